@@ -1,0 +1,182 @@
+/*
+ * lsgd.h — C ABI of liblsgd: the data-parallel hot path of one round of
+ * system-aware biased local SGD on a single NVIDIA B200 (sm_100a).
+ *
+ * The path has three parts (paper: Algorithm 1, Section 4.2, Section 4.3):
+ *   1. the per-sample loss record  — a softmax cross-entropy scorer that turns a
+ *      candidate pool's logits and labels into one loss per sample;
+ *   2. the deterministic loss-based top-k selection for the fast workers;
+ *   3. the biased model aggregation x_{t+1} = sum_i w_i * x^i_t   (Eq. 3).
+ *
+ * Conventions shared by every entry point
+ *   - "device" pointers are CUDA global-memory addresses on the CURRENT device;
+ *     "host" pointers are ordinary process memory.  Each argument says which.
+ *   - The caller owns every buffer, including the workspace.  The library
+ *     allocates no device memory, frees nothing and keeps no pointer after the
+ *     kernels it enqueued have run.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Calls only enqueue work on that stream and return; they do not
+ *     synchronise, except lsgd_read_device_status.
+ *   - Errors are reported by return value only.  Argument errors are found on
+ *     the host before anything is launched, so a failing call has no effect on
+ *     the device.  No kernel traps or spins without bound.
+ *   - A size of zero (N == 0, k == 0, D == 0) is legal: the call returns LSGD_OK
+ *     without launching anything.
+ *   - Workspaces must be 256-byte aligned.  Their contents are scratch: they
+ *     need no initialisation and have no meaning after the call, except for the
+ *     status block read by lsgd_read_device_status.
+ *   - Two calls that use the same workspace must be ordered on one stream.
+ */
+#ifndef LSGD_H_
+#define LSGD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(_WIN32)
+#define LSGD_API
+#else
+#define LSGD_API __attribute__((visibility("default")))
+#endif
+
+typedef enum lsgd_status {
+    LSGD_OK = 0,
+    LSGD_ERR_INVALID_ARG = 1, /* NULL where data is needed, negative size, k > N, P out of range, overlap */
+    LSGD_ERR_UNSUPPORTED = 2, /* a dtype / order value the library does not know, N >= 2^31          */
+    LSGD_ERR_ALIGNMENT = 3,   /* pointer not aligned to its element size, workspace not to 256 B      */
+    LSGD_ERR_WORKSPACE = 4,   /* ws_bytes smaller than the matching *_workspace_bytes query           */
+    LSGD_ERR_CUDA = 5,        /* the CUDA runtime refused a launch or a memset                        */
+    LSGD_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out (reported via the status block)   */
+} lsgd_status;
+
+/* Element type of the logits. Labels are always int64, losses always fp32. */
+typedef enum lsgd_dtype { LSGD_F32 = 0, LSGD_BF16 = 1 } lsgd_dtype;
+
+/* Order of the k selected indices.  Both orders are unique for a given input. */
+typedef enum lsgd_order {
+    LSGD_ORDER_LOSS_DESC = 0, /* highest loss first; equal losses by ascending index */
+    LSGD_ORDER_INDEX_ASC = 1  /* the same set, ascending index                       */
+} lsgd_order;
+
+/* Largest number of worker replicas one lsgd_aggregate call accepts. */
+#define LSGD_MAX_REPLICAS 64
+
+/* Library version as major*10000 + minor*100 + patch. */
+LSGD_API int lsgd_version(void);
+
+/* Static, NUL-terminated description of a status code (never NULL). */
+LSGD_API const char* lsgd_status_string(int status);
+
+/* ------------------------------------------------------------------------- */
+/* Workspace sizes (host-only arithmetic; 0 on invalid arguments).            */
+/* ------------------------------------------------------------------------- */
+LSGD_API size_t lsgd_score_workspace_bytes(int64_t N, int64_t T, int64_t C);
+LSGD_API size_t lsgd_topk_workspace_bytes(int64_t N, int64_t k);
+LSGD_API size_t lsgd_score_topk_workspace_bytes(int64_t N, int64_t T, int64_t C, int64_t k);
+
+/*
+ * lsgd_score_losses — the per-sample loss record of Algorithm 1 ("record all
+ * individual loss of processed data"; the stored value is one float per sample,
+ * Section 4.4 "Potential Limitations").  The loss f(x, xi) of the problem
+ * definition (Section 2) is taken to be softmax cross-entropy with natural log.
+ *
+ *   token loss   l[n,t] = -log softmax(logits[n,t,:])[labels[n,t]]
+ *   sample loss  losses[n] = mean of l[n,t] over the tokens t whose label is not
+ *                ignore_index, summed in a fixed order; 0 if every token of the
+ *                sample is ignored.  T == 1 is plain classification.
+ *
+ *   logits  device, [N, T, C] row-major, contiguous, dtype `dtype`, aligned to
+ *           its element size (16-byte alignment is faster, not required).
+ *           Values must be finite.  Rows whose label is ignore_index are not read.
+ *   labels  device, [N, T] int64.  A label outside [0, C) that is not
+ *           ignore_index makes that token's loss NaN (and so the sample's) and
+ *           is counted in the status block.
+ *   losses  device, [N] fp32, written in full.  Must not overlap logits.
+ *   ws      device workspace of at least lsgd_score_workspace_bytes(N, T, C).
+ *
+ * Arithmetic is fp32 (bf16 logits are widened exactly); results are within
+ * 1e-5 relative of an exact evaluation, also for losses near zero.
+ * Results do not depend on the launch geometry: same input, same bits.
+ */
+LSGD_API lsgd_status lsgd_score_losses(const void* logits, lsgd_dtype dtype, const int64_t* labels,
+                                       int64_t N, int64_t T, int64_t C, int64_t ignore_index,
+                                       float* losses, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * lsgd_topk_select — deterministic loss-based top-k selection (Section 4.2,
+ * "Data Allocation for Fast Workers"; Algorithm 1, the "select ... high-loss
+ * samples" step).  Selects the k entries that come first in the total order
+ *     higher loss first, then lower index,
+ * where -0.0 equals +0.0 and every NaN ranks above +inf (NaNs tie with each
+ * other).  Exact: integer comparisons only, bit-reproducible.
+ *
+ *   losses    device, [N] fp32.  N < 2^31: indices are 32-bit, as the index
+ *             payload quoted in Section 4.2 implies.
+ *   k         0 <= k <= N.
+ *   out_idx   device, [k] int32, the selected indices in `order`.
+ *   out_vals  device, [k] fp32 or NULL: losses[out_idx[j]], bits unchanged.
+ *   ws        device workspace of at least lsgd_topk_workspace_bytes(N, k).
+ */
+LSGD_API lsgd_status lsgd_topk_select(const float* losses, int64_t N, int64_t k, lsgd_order order,
+                                      int32_t* out_idx, float* out_vals, void* ws, size_t ws_bytes,
+                                      void* cuda_stream);
+
+/*
+ * lsgd_score_topk — lsgd_score_losses followed by lsgd_topk_select on its
+ * result, enqueued as one sequence in which the scorer's epilogue already
+ * builds the selector's first radix histogram.  `losses` ([N], device) is
+ * still written in full: it is the method's loss table.  Arguments as in the
+ * two calls above; ws >= lsgd_score_topk_workspace_bytes(N, T, C, k).
+ * Bit-identical to calling the two entry points one after the other.
+ */
+LSGD_API lsgd_status lsgd_score_topk(const void* logits, lsgd_dtype dtype, const int64_t* labels,
+                                     int64_t N, int64_t T, int64_t C, int64_t ignore_index, int64_t k,
+                                     lsgd_order order, float* losses, int32_t* out_idx, float* out_vals,
+                                     void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * lsgd_aggregate — biased model aggregation, Eq. 3:  out[j] = sum_i w_i * x_i[j]
+ * over the P worker replicas' flattened parameters, accumulated in fp32 in
+ * ascending i (one multiply, then fused multiply-adds).  Every replica element
+ * is read exactly once.
+ *
+ *   replicas  HOST array of P DEVICE pointers, each to D fp32 values, 4-byte
+ *             aligned (16-byte alignment of all P pointers and of `out` takes
+ *             the vectorised path).  Read before the call returns.
+ *   weights   HOST array of P fp32 weights, read before the call returns, used
+ *             exactly as given: not normalised, not clamped (Remark 2: any
+ *             weight vector is admissible).  w_i == 0 does not skip replica i
+ *             (IEEE rules: 0 * inf = NaN).
+ *   P         1 <= P <= LSGD_MAX_REPLICAS.      D >= 0.
+ *   out       device, [D] fp32.  May be exactly one of the replicas (in-place
+ *             update); any other overlap with a replica is LSGD_ERR_INVALID_ARG.
+ */
+LSGD_API lsgd_status lsgd_aggregate(const float* const* replicas, const float* weights, int32_t P,
+                                    int64_t D, float* out, void* cuda_stream);
+
+/*
+ * lsgd_weights_from_steps — the weights of Eq. 3, w_i = tau_i / sum_j tau_j, from
+ * the local step counts tau_i of the P workers.  Host only; computed in double
+ * and rounded once to fp32.  tau_i >= 0 and sum > 0, else LSGD_ERR_INVALID_ARG.
+ *   tau    host, [P] int32        w_out  host, [P] fp32
+ */
+LSGD_API lsgd_status lsgd_weights_from_steps(const int32_t* tau, int32_t P, float* w_out);
+
+/*
+ * lsgd_read_device_status — reads the status block that the last scoring or
+ * selection call left at the start of `ws`.  Synchronises `cuda_stream`.
+ *   bad_label_count  host, out: tokens whose label was outside [0, C) and not
+ *                    ignore_index in that call.
+ * Returns LSGD_ERR_TIMEOUT if a bounded device-side wait ran out in that call,
+ * LSGD_ERR_CUDA if the copy failed, else LSGD_OK.
+ */
+LSGD_API lsgd_status lsgd_read_device_status(const void* ws, int32_t* bad_label_count, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LSGD_H_ */
