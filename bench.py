@@ -1,0 +1,400 @@
+#!/usr/bin/env python
+"""Benchmark of the biased-local-SGD hot path on B200.
+
+One "step" is one pass of the whole hot path over one synthetic round:
+    lsgd_score_topk  (per-sample loss record + deterministic top-k, Section 4.2)
+    lsgd_aggregate   (Eq. 3)
+with the step-count weights of Eq. 3 computed once by lsgd_weights_from_steps
+where the round uses them.  Inputs are resident in HBM for `value`; the `e2e`
+leg repeats the step with host->device copies of all inputs from pinned memory
+and device->host copies of the results inside the timed region.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead
+(bounded samples of the same workload on the host cores).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2508_08540_b200 import workloads as wl  # noqa: E402
+
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(p))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (no MEASURED_PEAKS.json)"
+
+
+# --------------------------------------------------------------------------- #
+# algorithmic bytes
+# --------------------------------------------------------------------------- #
+def score_topk_bytes(cfg, labels: np.ndarray) -> int:
+    """Logits of the unmasked rows + every label + the loss table in and out of the selector + k indices and values."""
+    es = 4 if cfg.dtype == "f32" else 2
+    unmasked = int((labels != wl.IGNORE_INDEX).sum())
+    rows = labels.size
+    b = unmasked * (cfg.C * es + 4) + rows * 8
+    b += 4 * cfg.N + 4 * cfg.N + 8 * cfg.k
+    return b
+
+
+def aggregate_bytes(cfg) -> int:
+    return 4 * cfg.D * (cfg.P + 1)
+
+
+# --------------------------------------------------------------------------- #
+# clocks (read-only NVML sampling while the timed region runs)
+# --------------------------------------------------------------------------- #
+class ClockSampler:
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.sm_max = [], set(), None
+        self._stop = threading.Event()
+        self._t = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+        self.period = period_s
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+                 "hw_power_brake_slowdown": 0x80, "applications_clocks_setting": 0x2, "sync_boost": 0x10}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv:
+            self._t = threading.Thread(target=self._run, daemon=True)
+            self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._t:
+            self._t.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": ["unavailable"]}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.sm_max, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------- #
+# CPU oracle timing (bounded samples)
+# --------------------------------------------------------------------------- #
+def oracle_sample(cfg, n_samples: int, d_elems: int):
+    """Inputs for an oracle run on the first n_samples samples and the first d_elems parameters."""
+    x, y = wl.pool_rows(cfg, 0, n_samples)
+    reps = [wl.replica_slice(cfg, i, 0, d_elems) for i in range(cfg.P)]
+    return x, y, reps
+
+
+def round_weights_oracle(cfg, oracle):
+    return oracle.weights_from_steps(wl.step_counts(cfg)) if cfg.weight_mode == "steps" else wl.weight_draws(cfg)
+
+
+def time_oracle_step(oracle, cfg, x, y, reps, w):
+    n = x.shape[0]
+    k = max(1, min(n, round(cfg.k * n / cfg.N)))
+    t0 = time.perf_counter()
+    loss, _ = oracle.score(x, y)
+    oracle.topk(loss.astype(np.float32), k, oracle.LOSS_DESC)
+    t1 = time.perf_counter()
+    oracle.aggregate(reps, w)
+    t2 = time.perf_counter()
+    return t1 - t0, t2 - t1
+
+
+def calibrate_oracle(oracle, cfg, budget_s: float):
+    """Sample sizes (samples, parameters) whose oracle run takes about budget_s (2/3 scoring, 1/3 aggregation)."""
+    n0 = max(1, min(cfg.N, 4096 // max(1, cfg.T * cfg.C // 1000 + 1)))
+    d0 = min(cfg.D, 1 << 18)
+    x, y, reps = oracle_sample(cfg, n0, d0)
+    w = round_weights_oracle(cfg, oracle)
+    ts, ta = time_oracle_step(oracle, cfg, x, y, reps, w)
+    n = int(max(1, min(cfg.N, n0 * (budget_s * 2 / 3) / max(ts, 1e-6))))
+    d = int(max(1024, min(cfg.D, d0 * (budget_s / 3) / max(ta, 1e-6))))
+    return n, d
+
+
+def cpu_baseline(cfg, budget_s: float = 12.0):
+    from oracle import oracle
+
+    oracle.build()
+    n, d = calibrate_oracle(oracle, cfg, budget_s)
+    x, y, reps = oracle_sample(cfg, n, d)
+    w = round_weights_oracle(cfg, oracle)
+    ts, ta = time_oracle_step(oracle, cfg, x, y, reps, w)
+    return {
+        "value": n / ts, "unit": "samples/s", "cores": 1, "kind": "oracle",
+        "sample": f"first {n} of {cfg.N} samples scored + top-k of them; aggregation of the first {d} of {cfg.D} parameters "
+                  f"of all {cfg.P} replicas",
+        "score_topk_s": ts, "aggregate_s": ta, "aggregate_gbs": 4 * d * (cfg.P + 1) / ta / 1e9,
+        "host_cores_available": os.cpu_count(),
+    }
+
+
+def run_reference(args, cfg):
+    """--impl reference: the CPU oracle, as it stands, on bounded samples of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle
+
+    oracle.build()
+    per_step = max(0.05, min(10.0, 90.0 / (args.steps + args.warmup)))
+    n, d = calibrate_oracle(oracle, cfg, per_step)
+    x, y, reps = oracle_sample(cfg, n, d)
+    w = round_weights_oracle(cfg, oracle)
+    for _ in range(args.warmup):
+        time_oracle_step(oracle, cfg, x, y, reps, w)
+    ts = ta = 0.0
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        a, b = time_oracle_step(oracle, cfg, x, y, reps, w)
+        ts += a
+        ta += b
+    total = time.perf_counter() - t0
+    value = n * args.steps / ts
+    sample = (f"each step: first {n} of {cfg.N} samples scored + top-k of them, aggregation of the first {d} of {cfg.D} "
+              f"parameters of all {cfg.P} replicas")
+    line = {
+        "impl": "reference", "metric": "score+top-k samples/s", "value": value, "unit": "samples/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg, "host memory; CPU oracle"),
+        "aggregation": {"value": 4 * d * (cfg.P + 1) * args.steps / ta / 1e9, "unit": "GB/s"},
+        "cpu_baseline": {"value": value, "unit": "samples/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "samples/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg, residency: str):
+    return {
+        "workload": f"config {cfg.cfg_id} ({cfg.name}-scale round): pool {cfg.N} x {cfg.T} x {cfg.C} {cfg.dtype} logits, "
+                    f"k={cfg.k}; {cfg.P} replicas x {cfg.D} fp32 parameters",
+        "N": cfg.N, "T": cfg.T, "C": cfg.C, "k": cfg.k, "P": cfg.P, "D": cfg.D, "order": "loss_desc",
+        "l2": "inputs larger than L2 (no flush needed)" if cfg.logit_bytes > (1 << 28) else "L2 flushed between steps",
+        "inputs": residency,
+    }
+
+
+# --------------------------------------------------------------------------- #
+# GPU arm
+# --------------------------------------------------------------------------- #
+def run_gpu(args, cfg):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2508_08540_b200 import lsgd
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    lsgd.lib()
+
+    # ---- inputs: generated on the host into pinned memory, then made resident
+    t_gen = time.perf_counter()
+    tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    h_logits = torch.empty((cfg.N, cfg.T, cfg.C), dtype=tdt, pin_memory=True)
+    h_labels = torch.empty((cfg.N, cfg.T), dtype=torch.int64, pin_memory=True)
+    np_logits = h_logits.view(torch.int16).numpy().view(np.uint16) if cfg.dtype == "bf16" else h_logits.numpy()
+    step = max(1, (1 << 28) // max(1, cfg.T * cfg.C * np_logits.itemsize))
+    for s0 in range(0, cfg.N, step):
+        s1 = min(cfg.N, s0 + step)
+        x, y = wl.pool_rows(cfg, s0, s1)
+        np_logits[s0:s1] = x
+        h_labels.numpy()[s0:s1] = y
+    h_reps = [torch.empty(cfg.D, dtype=torch.float32, pin_memory=True) for _ in range(cfg.P)]
+    for i in range(cfg.P):
+        wl.replica_slice(cfg, i, out=h_reps[i].numpy())
+    if cfg.weight_mode == "steps":
+        weights = lsgd.weights_from_steps(wl.step_counts(cfg).tolist())
+    else:
+        weights = wl.weight_draws(cfg).tolist()
+    gen_s = time.perf_counter() - t_gen
+
+    d_logits = h_logits.to(dev, non_blocking=True)
+    d_labels = h_labels.to(dev, non_blocking=True)
+    d_reps = [r.to(dev, non_blocking=True) for r in h_reps]
+    losses = torch.empty(cfg.N, dtype=torch.float32, device=dev)
+    idx = torch.empty(cfg.k, dtype=torch.int32, device=dev)
+    vals = torch.empty(cfg.k, dtype=torch.float32, device=dev)
+    out = torch.empty(cfg.D, dtype=torch.float32, device=dev)
+    ws = lsgd.workspace(lsgd.score_topk_workspace_bytes(cfg.N, cfg.T, cfg.C, cfg.k), dev)
+    flush = None if cfg.logit_bytes > (1 << 28) else torch.empty(1 << 28, dtype=torch.uint8, device=dev)
+    torch.cuda.synchronize()
+
+    def step_resident(ev=None):
+        if flush is not None:
+            flush.fill_(1)
+        if ev:
+            ev[0].record()
+        lsgd.score_topk(d_logits, d_labels, cfg.k, lsgd.ORDER_LOSS_DESC, losses=losses, out_idx=idx, out_vals=vals, ws=ws)
+        if ev:
+            ev[1].record()
+        lsgd.aggregate(d_reps, weights, out=out)
+        if ev:
+            ev[2].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step_resident()
+    barrier()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        barrier()
+        start.record()
+        for i in range(args.steps):
+            step_resident(evs[i])
+        end.record()
+        barrier()
+    total_ms = start.elapsed_time(end)
+    st_ms = np.array([e[0].elapsed_time(e[1]) for e in evs])
+    ag_ms = np.array([e[1].elapsed_time(e[2]) for e in evs])
+    bad = lsgd.read_device_status(ws)
+
+    # ---- end to end: inputs from pinned host memory, results back to the host, every step
+    e2e_steps = max(1, min(args.steps, 5 if cfg.logit_bytes > (1 << 30) else 20))
+    h_idx = torch.empty(cfg.k, dtype=torch.int32, pin_memory=True)
+    h_vals = torch.empty(cfg.k, dtype=torch.float32, pin_memory=True)
+    h_out = torch.empty(cfg.D, dtype=torch.float32, pin_memory=True)
+    h2d = h_logits.numel() * h_logits.element_size() + h_labels.numel() * 8 + cfg.P * cfg.D * 4
+    d2h = cfg.k * 8 + cfg.D * 4
+
+    def step_e2e():
+        d_logits.copy_(h_logits, non_blocking=True)
+        d_labels.copy_(h_labels, non_blocking=True)
+        for d, h in zip(d_reps, h_reps):
+            d.copy_(h, non_blocking=True)
+        lsgd.score_topk(d_logits, d_labels, cfg.k, lsgd.ORDER_LOSS_DESC, losses=losses, out_idx=idx, out_vals=vals, ws=ws)
+        lsgd.aggregate(d_reps, weights, out=out)
+        h_idx.copy_(idx, non_blocking=True)
+        h_vals.copy_(vals, non_blocking=True)
+        h_out.copy_(out, non_blocking=True)
+
+    step_e2e()
+    barrier()
+    s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s2.record()
+    for _ in range(e2e_steps):
+        step_e2e()
+    e2.record()
+    barrier()
+    e2e_ms = s2.elapsed_time(e2)
+
+    t = torch.tensor([total_ms, float(st_ms.sum()), float(ag_ms.sum()), e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, st_sum, ag_sum, e2e_ms = t.tolist()
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        st_bytes = score_topk_bytes(cfg, h_labels.numpy())
+        ag_bytes = aggregate_bytes(cfg)
+        st_gbs = st_bytes * args.steps / (st_sum * 1e-3) / 1e9
+        ag_gbs = ag_bytes * args.steps / (ag_sum * 1e-3) / 1e9
+        n_launch = launches_per_step(cfg)
+        line = {
+            "metric": "score+top-k samples/s", "value": world * cfg.N * args.steps / (st_sum * 1e-3), "unit": "samples/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(cfg, "resident in HBM"),
+            "score_topk": {"ms": st_sum / args.steps, "ms_best": float(st_ms.min()), "gbs": st_gbs,
+                           "frac_of_measured_hbm": st_gbs / peak, "frac_of_nominal_8tbs": st_gbs / NOMINAL_HBM_GBS,
+                           "algorithmic_bytes": st_bytes, "bad_labels": bad},
+            "aggregation": {"value": world * ag_gbs, "unit": "GB/s", "ms": ag_sum / args.steps, "ms_best": float(ag_ms.min()),
+                            "frac_of_measured_hbm": ag_gbs / peak, "frac_of_nominal_8tbs": ag_gbs / NOMINAL_HBM_GBS,
+                            "algorithmic_bytes": ag_bytes},
+            "round_samples_per_s": world * cfg.N * args.steps / (total_ms * 1e-3),
+            "roofline": {"bound": "hbm", "kernel": "lsgd_score_topk (scorer kernel + memset, sequence mean, selector)",
+                         "achieved": st_gbs, "peak": peak, "unit": "GB/s", "frac": st_gbs / peak, "traffic": None,
+                         "peak_source": peak_src},
+            "roofline_aggregate": {"bound": "hbm", "kernel": "aggregate_vec4_kernel", "achieved": ag_gbs, "peak": peak,
+                                   "unit": "GB/s", "frac": ag_gbs / peak, "traffic": None, "peak_source": peak_src},
+            "e2e": {"value": world * cfg.N * e2e_steps / (e2e_ms * 1e-3), "unit": "samples/s", "ms_per_step": e2e_ms / e2e_steps,
+                    "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "note": "whole step (score+top-k and aggregation) incl. copies; bound by the host link"},
+            "gpu_launches": n_launch * args.steps,
+            "clocks": clocks.summary(),
+            "input_generation_s": gen_s,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(cfg)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def launches_per_step(cfg) -> int:
+    """Kernels of liblsgd launched by one step (memsets excluded), from the launch logic of the library."""
+    n = 1 + (1 if cfg.T > 1 else 0)                # scorer (+ sequence mean)
+    if cfg.N <= 4096:
+        n += 1                                      # single-CTA selector
+    else:
+        n += 2 + 1 + 1 + 4                          # two more histogram passes, count, emit, four sort passes
+    n += 1 + (1 if cfg.D % 4 else 0)                # aggregation (+ ragged tail)
+    return n
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=4, choices=sorted(wl.CONFIGS))
+    ap.add_argument("--impl", default="lsgd", choices=["lsgd", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = wl.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_gpu(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,103 @@
+// Internal declarations shared by the translation units of liblsgd.
+// Nothing here is part of the C ABI (see include/lsgd.h for that).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lsgd.h"
+
+namespace lsgd {
+
+// ---------------------------------------------------------------------------
+// Status block: the first 256 bytes of every scoring / selection workspace.
+// Zeroed (together with the selector's histograms) by one memset per call.
+// ---------------------------------------------------------------------------
+struct StatusBlock {
+    int32_t bad_labels;   // tokens with a label outside [0, C) that is not ignore_index
+    int32_t timeout;      // set when a bounded device-side wait ran out
+    uint32_t row_ticket;  // dynamic row scheduler of the large-row scorer
+    uint32_t pad[61];
+};
+static_assert(sizeof(StatusBlock) == 256, "status block is 256 bytes");
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// ---------------------------------------------------------------------------
+// Selector geometry.  Keys are order-preserving 32-bit images of the losses,
+// resolved in three radix digits of 11, 11 and 10 bits, most significant first.
+// ---------------------------------------------------------------------------
+constexpr int kSelPasses = 3;
+constexpr int kSelBins = 2048;            // 11-bit digits (the last digit uses 1024 of them)
+constexpr int kTile = 4096;               // elements per CTA in the count / emit / sort kernels
+constexpr int kSmallN = 4096;             // pools up to this size are sorted by one CTA in shared memory
+constexpr int kSortBins = 256;            // 8-bit digits of the stable LSD sort of the selected pairs
+
+struct TopkWorkspace {       // device pointers carved out of the caller's workspace
+    StatusBlock* status;
+    uint32_t* hist;          // [kSelPasses][kSelBins]
+    uint32_t* tile_counts;   // [tiles(N)][2]  (#keys above the threshold, #keys equal to it)
+    uint32_t* keys[2];       // [k] ping-pong: keys of the selected entries
+    int32_t* idx[2];         // [k] ping-pong: their indices
+    uint32_t* tile_hist;     // [tiles(k)][kSortBins] digit counts per tile of the current sort pass
+};
+
+struct ScoreWorkspace {
+    StatusBlock* status;
+    float* token_loss;       // [N*T] when T > 1, else unused
+};
+
+size_t topk_workspace_bytes(int64_t N, int64_t k);
+size_t score_workspace_bytes(int64_t N, int64_t T, int64_t C);
+TopkWorkspace carve_topk(void* ws, int64_t N, int64_t k);
+ScoreWorkspace carve_score(void* ws, int64_t N, int64_t T, int64_t C);
+// Clears the status block, the selector's histograms and the sort's digit counts.
+cudaError_t zero_topk_workspace(void* ws, int64_t k, cudaStream_t s);
+
+// Launchers (each returns the CUDA error of its launches).  `hist0` non-NULL asks
+// the scorer to accumulate the selector's first-digit histogram while it writes
+// the losses.
+cudaError_t launch_aggregate(const float* const* replicas, const float* weights, int P, int64_t D, float* out,
+                             bool vector_ok, cudaStream_t s);
+cudaError_t launch_score(const void* logits, lsgd_dtype dt, const int64_t* labels, int64_t N, int64_t T, int64_t C,
+                         int64_t ignore_index, float* losses, const ScoreWorkspace& ws, uint32_t* hist0,
+                         cudaStream_t s);
+cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order order, int32_t* out_idx,
+                        float* out_vals, const TopkWorkspace& ws, bool hist0_ready, cudaStream_t s);
+
+int sm_count();  // multiprocessors of the current device (cached per device)
+
+// ---------------------------------------------------------------------------
+// Device helpers
+// ---------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+// Order-preserving key of a loss: larger key = selected earlier.  -0 maps to +0,
+// every NaN maps to the largest key (it ranks above +inf).
+__device__ __forceinline__ uint32_t loss_key(float v) {
+    uint32_t u = __float_as_uint(v);
+    if (v != v) return 0xFFFFFFFFu;
+    if (u == 0x80000000u) u = 0u;
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace lsgd

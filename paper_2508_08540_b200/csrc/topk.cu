@@ -1,0 +1,485 @@
+// Deterministic loss-based top-k selection (Section 4.2, "Data Allocation for
+// Fast Workers": the highest-loss samples go to the fast workers).
+//
+// Total order: higher loss first, then lower index.  Losses are mapped to
+// order-preserving 32-bit keys (loss_key), so everything below is integer work
+// and the result is exact and bit-reproducible.
+//
+//   1. radix select: three histogram passes (11 + 11 + 10 bits, most significant
+//      digit first) find the key T of the k-th entry and r, the number of entries
+//      equal to T that still belong to the selection;
+//   2. ordered compaction: per-tile counts, then an emit pass that keeps every
+//      key > T and the r lowest-index keys == T, writing them in index order
+//      (scan-based positions: no atomics decide an order);
+//   3. for loss-descending output, a stable LSD radix sort (four 8-bit digits) of
+//      the k (key, index) pairs; stability turns the index-ascending input order
+//      into the required tie-break.  Each scatter pass accumulates the digit
+//      counts of the next pass, so the sort is one kernel per digit.
+// Pools of at most kSmallN entries are sorted whole by a single CTA instead.
+#include <algorithm>
+
+#include "lsgd_internal.cuh"
+
+namespace lsgd {
+
+size_t topk_workspace_bytes(int64_t N, int64_t k) {
+    if (N < 0 || k < 0 || k > N) return 0;
+    const size_t tiles_n = static_cast<size_t>((N + kTile - 1) / kTile);
+    const size_t tiles_k = static_cast<size_t>((k + kTile - 1) / kTile);
+    size_t b = sizeof(StatusBlock);
+    b += align_up(sizeof(uint32_t) * kSelPasses * kSelBins);
+    b += align_up(sizeof(uint32_t) * 4 * tiles_k * kSortBins);
+    b += align_up(sizeof(uint32_t) * 2 * tiles_n);
+    b += 4 * align_up(sizeof(uint32_t) * static_cast<size_t>(k));
+    return b;
+}
+
+// Bytes at the start of the workspace that one memset must clear before a call.
+static size_t topk_zero_bytes(int64_t k) {
+    const size_t tiles_k = static_cast<size_t>((k + kTile - 1) / kTile);
+    return sizeof(StatusBlock) + align_up(sizeof(uint32_t) * kSelPasses * kSelBins) +
+           align_up(sizeof(uint32_t) * 4 * tiles_k * kSortBins);
+}
+
+TopkWorkspace carve_topk(void* ws, int64_t N, int64_t k) {
+    const size_t tiles_n = static_cast<size_t>((N + kTile - 1) / kTile);
+    const size_t tiles_k = static_cast<size_t>((k + kTile - 1) / kTile);
+    unsigned char* p = static_cast<unsigned char*>(ws);
+    TopkWorkspace w;
+    w.status = reinterpret_cast<StatusBlock*>(p);
+    p += sizeof(StatusBlock);
+    w.hist = reinterpret_cast<uint32_t*>(p);
+    p += align_up(sizeof(uint32_t) * kSelPasses * kSelBins);
+    w.tile_hist = reinterpret_cast<uint32_t*>(p);
+    p += align_up(sizeof(uint32_t) * 4 * tiles_k * kSortBins);
+    w.tile_counts = reinterpret_cast<uint32_t*>(p);
+    p += align_up(sizeof(uint32_t) * 2 * tiles_n);
+    const size_t kb = align_up(sizeof(uint32_t) * static_cast<size_t>(k));
+    w.keys[0] = reinterpret_cast<uint32_t*>(p);
+    w.keys[1] = reinterpret_cast<uint32_t*>(p + kb);
+    w.idx[0] = reinterpret_cast<int32_t*>(p + 2 * kb);
+    w.idx[1] = reinterpret_cast<int32_t*>(p + 3 * kb);
+    return w;
+}
+
+cudaError_t zero_topk_workspace(void* ws, int64_t k, cudaStream_t s) {
+    return cudaMemsetAsync(ws, 0, topk_zero_bytes(k), s);
+}
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kPerThread = kTile / kThreads;  // 16
+
+__device__ __forceinline__ uint32_t digit_of(uint32_t key, int pass) {
+    return pass == 0 ? key >> 21 : pass == 1 ? (key >> 10) & 0x7FFu : key & 0x3FFu;
+}
+
+// Block-wide exclusive scan of one value per thread (kThreads threads).
+// `scratch` holds kThreads / 32 + 1 words.  Returns the exclusive prefix; the
+// block total is left in scratch[kThreads / 32].
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* scratch) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    __syncthreads();  // scratch may still be read from an earlier call
+    if (lane == 31) scratch[warp] = inc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t run = 0;
+        for (int w = 0; w < kThreads / 32; ++w) {
+            const uint32_t c = scratch[w];
+            scratch[w] = run;
+            run += c;
+        }
+        scratch[kThreads / 32] = run;
+    }
+    __syncthreads();
+    return scratch[warp] + inc - v;
+}
+
+// Walks a histogram from its highest bin down and finds the bin that holds the
+// `want`-th entry (1-based).  On return (all threads): bin, and `want` reduced by
+// the entries in the bins above it.
+__device__ void find_bin(const uint32_t* hist, int nbins, uint32_t& want, uint32_t& bin, uint32_t* scratch,
+                         uint32_t* result) {
+    const int per = nbins / kThreads;  // 8 or 4
+    // thread t owns bins [nbins - 1 - t*per - (per - 1), nbins - 1 - t*per], highest first
+    uint32_t c[8];
+    uint32_t sum = 0;
+    for (int i = 0; i < per; ++i) {
+        c[i] = hist[nbins - 1 - (threadIdx.x * per + i)];
+        sum += c[i];
+    }
+    const uint32_t before = block_exclusive_scan(sum, scratch);
+    if (before < want && want <= before + sum) {
+        uint32_t run = before;
+        for (int i = 0; i < per; ++i) {
+            if (want <= run + c[i]) {
+                result[0] = nbins - 1 - (threadIdx.x * per + i);
+                result[1] = want - run;
+                break;
+            }
+            run += c[i];
+        }
+    }
+    __syncthreads();
+    bin = result[0];
+    want = result[1];
+    __syncthreads();
+}
+
+// Resolves the digits of the threshold key that passes [0, upto) fixed.
+// Returns the key prefix (digits placed, lower bits zero) and the rank left
+// inside that prefix.
+__device__ uint32_t resolve_prefix(const uint32_t* hist, int upto, uint32_t k, uint32_t& want, uint32_t* scratch,
+                                   uint32_t* result) {
+    uint32_t prefix = 0;
+    want = k;
+    for (int p = 0; p < upto; ++p) {
+        uint32_t bin;
+        find_bin(hist + p * kSelBins, p == 2 ? 1024 : kSelBins, want, bin, scratch, result);
+        prefix |= p == 0 ? bin << 21 : p == 1 ? bin << 10 : bin;
+    }
+    return prefix;
+}
+
+__device__ __forceinline__ uint32_t prefix_mask(int pass) { return pass == 0 ? 0u : pass == 1 ? 0xFFE00000u : 0xFFFFFC00u; }
+
+// Loads the 16 keys thread `threadIdx.x` owns in tile `tile` (consecutive
+// indices), 0 beyond N.  Key 0 belongs to no loss (loss_key never returns it).
+__device__ __forceinline__ void load_keys(const float* __restrict__ losses, int64_t N, int64_t base, uint32_t (&key)[kPerThread]) {
+#pragma unroll
+    for (int i = 0; i < kPerThread; ++i) {
+        const int64_t j = base + i;
+        key[i] = j < N ? loss_key(losses[j]) : 0u;
+    }
+}
+
+// Histogram pass `pass`: counts digit `pass` of the keys that match the prefix
+// fixed by the earlier passes.
+__global__ void __launch_bounds__(kThreads)
+select_hist_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, int pass, uint32_t* hist) {
+    __shared__ uint32_t hist_s[kSelBins];
+    __shared__ uint32_t scratch[kThreads / 32 + 1];
+    __shared__ uint32_t result[2];
+    for (int i = threadIdx.x; i < kSelBins; i += kThreads) hist_s[i] = 0;
+    uint32_t want;
+    const uint32_t prefix = resolve_prefix(hist, pass, k, want, scratch, result);
+    __syncthreads();
+    const uint32_t mask = prefix_mask(pass);
+    for (int64_t tile = blockIdx.x; tile * kTile < N; tile += gridDim.x) {
+        const int64_t base = tile * kTile;
+#pragma unroll 4
+        for (int i = 0; i < kPerThread; ++i) {
+            const int64_t j = base + i * kThreads + threadIdx.x;
+            if (j < N) {
+                const uint32_t key = loss_key(losses[j]);
+                if ((key & mask) == prefix) atomicAdd(&hist_s[digit_of(key, pass)], 1u);
+            }
+        }
+    }
+    __syncthreads();
+    uint32_t* out = hist + pass * kSelBins;
+    for (int i = threadIdx.x; i < kSelBins; i += kThreads)
+        if (hist_s[i]) atomicAdd(&out[i], hist_s[i]);
+}
+
+// Per tile: how many keys are above the threshold, how many equal it.
+__global__ void __launch_bounds__(kThreads)
+select_count_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, const uint32_t* hist,
+                    uint32_t* tile_counts) {
+    __shared__ uint32_t scratch[kThreads / 32 + 1];
+    __shared__ uint32_t result[2];
+    __shared__ uint32_t cnt[2];
+    uint32_t want;
+    const uint32_t T = resolve_prefix(hist, kSelPasses, k, want, scratch, result);
+    for (int64_t tile = blockIdx.x; tile * kTile < N; tile += gridDim.x) {
+        if (threadIdx.x < 2) cnt[threadIdx.x] = 0;
+        __syncthreads();
+        uint32_t gt = 0, eq = 0;
+#pragma unroll 4
+        for (int i = 0; i < kPerThread; ++i) {
+            const int64_t j = tile * kTile + i * kThreads + threadIdx.x;
+            if (j < N) {
+                const uint32_t key = loss_key(losses[j]);
+                gt += key > T;
+                eq += key == T;
+            }
+        }
+        gt = warp_sum(static_cast<int>(gt));
+        eq = warp_sum(static_cast<int>(eq));
+        if ((threadIdx.x & 31) == 0) {
+            atomicAdd(&cnt[0], gt);
+            atomicAdd(&cnt[1], eq);
+        }
+        __syncthreads();
+        if (threadIdx.x < 2) tile_counts[2 * tile + threadIdx.x] = cnt[threadIdx.x];
+        __syncthreads();
+    }
+}
+
+// Emit: keeps every key above the threshold and the first `r` (by index) equal
+// to it, in index order.  Positions come from the tile counts and an in-tile
+// scan.  DIRECT: write the final index-ascending result; otherwise write the
+// (key, index) pairs for the sort and count their first sort digit.
+template <bool DIRECT>
+__global__ void __launch_bounds__(kThreads)
+select_emit_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, const uint32_t* hist,
+                   const uint32_t* __restrict__ tile_counts, int32_t* __restrict__ out_idx,
+                   float* __restrict__ out_vals, uint32_t* __restrict__ out_keys, uint32_t* __restrict__ tile_hist) {
+    __shared__ uint32_t scratch[kThreads / 32 + 1];
+    __shared__ uint32_t result[2];
+    __shared__ uint32_t pre[2];
+    uint32_t r;
+    const uint32_t T = resolve_prefix(hist, kSelPasses, k, r, scratch, result);
+    for (int64_t tile = blockIdx.x; tile * kTile < N; tile += gridDim.x) {
+        // entries above / equal to the threshold in the tiles before this one
+        if (threadIdx.x < 2) pre[threadIdx.x] = 0;
+        __syncthreads();
+        uint32_t gt = 0, eq = 0;
+        for (int64_t t = threadIdx.x; t < tile; t += kThreads) {
+            gt += tile_counts[2 * t];
+            eq += tile_counts[2 * t + 1];
+        }
+        gt = warp_sum(static_cast<int>(gt));
+        eq = warp_sum(static_cast<int>(eq));
+        if ((threadIdx.x & 31) == 0) {
+            atomicAdd(&pre[0], gt);
+            atomicAdd(&pre[1], eq);
+        }
+        __syncthreads();
+        const uint32_t gt_before = pre[0], eq_before = pre[1];
+
+        const int64_t base = tile * kTile + static_cast<int64_t>(threadIdx.x) * kPerThread;
+        uint32_t key[kPerThread];
+        load_keys(losses, N, base, key);
+        uint32_t my_gt = 0, my_eq = 0;
+#pragma unroll
+        for (int i = 0; i < kPerThread; ++i) {
+            my_gt += key[i] > T;
+            my_eq += (key[i] == T);
+        }
+        // one scan for both counts: each is at most kTile = 4096 < 2^16
+        const uint32_t packed = block_exclusive_scan(my_gt | (my_eq << 16), scratch);
+        uint32_t gt_run = gt_before + (packed & 0xFFFFu);
+        uint32_t eq_run = eq_before + (packed >> 16);
+#pragma unroll
+        for (int i = 0; i < kPerThread; ++i) {
+            const bool above = key[i] > T;
+            const bool tie = key[i] == T;
+            if (above || (tie && eq_run < r)) {
+                const uint32_t pos = gt_run + min(eq_run, r);
+                const int64_t j = base + i;
+                if (DIRECT) {
+                    out_idx[pos] = static_cast<int32_t>(j);
+                    if (out_vals) out_vals[pos] = losses[j];
+                } else {
+                    out_idx[pos] = static_cast<int32_t>(j);
+                    out_keys[pos] = key[i];
+                    atomicAdd(&tile_hist[(pos / kTile) * kSortBins + (255u - (key[i] & 0xFFu))], 1u);
+                }
+            }
+            gt_run += above;
+            eq_run += tie;
+        }
+        __syncthreads();
+    }
+}
+
+// One stable LSD pass over the selected pairs, on digit `pass` (8 bits, least
+// significant first), larger digits first.  Reads the digit counts per source
+// tile, ranks the tile's entries stably (warp match + per-warp counters), and
+// scatters.  Unless LAST, also counts the next digit per destination tile.
+template <bool LAST>
+__global__ void __launch_bounds__(kThreads)
+sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restrict__ idx_in, uint32_t k, int pass,
+                    const uint32_t* __restrict__ tile_hist, uint32_t* __restrict__ keys_out,
+                    int32_t* __restrict__ idx_out, uint32_t* __restrict__ next_hist,
+                    const float* __restrict__ losses, float* __restrict__ out_vals) {
+    constexpr int kWarps = kThreads / 32;
+    constexpr int kRounds = kTile / kThreads;  // 16 rounds of 32 consecutive entries per warp
+    __shared__ uint32_t counters[kWarps][kSortBins];
+    __shared__ uint32_t base_s[kSortBins];
+    __shared__ uint32_t scratch[kThreads / 32 + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t tiles = (k + kTile - 1) / kTile;
+    const int shift = 8 * pass;
+    for (uint32_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        // where each digit's run starts for this tile: all entries of earlier digits, plus
+        // this digit's entries in earlier tiles
+        {
+            const int d = threadIdx.x;  // kThreads == kSortBins
+            uint32_t total = 0, before = 0;
+            for (uint32_t t = 0; t < tiles; ++t) {
+                const uint32_t c = tile_hist[t * kSortBins + d];
+                total += c;
+                before += t < tile ? c : 0u;
+            }
+            const uint32_t excl = block_exclusive_scan(total, scratch);
+            base_s[d] = excl + before;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) counters[w][d] = 0;
+        }
+        __syncthreads();
+        uint32_t key[kRounds], rank[kRounds];
+        int32_t idx[kRounds];
+        const uint32_t first = tile * kTile + warp * (kRounds * 32);
+#pragma unroll
+        for (int rd = 0; rd < kRounds; ++rd) {
+            const uint32_t e = first + rd * 32 + lane;
+            const bool live = e < k;
+            key[rd] = live ? keys_in[e] : 0u;
+            idx[rd] = live ? idx_in[e] : 0;
+            const uint32_t dd = live ? 255u - ((key[rd] >> shift) & 0xFFu) : 256u;
+            const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dd);
+            const int leader = __ffs(peers) - 1;
+            uint32_t old = 0;
+            if (live && lane == leader) {
+                old = counters[warp][dd];
+                counters[warp][dd] = old + __popc(peers);
+            }
+            old = __shfl_sync(0xFFFFFFFFu, old, leader);
+            rank[rd] = old + __popc(peers & ((1u << lane) - 1u));
+            __syncwarp();
+        }
+        __syncthreads();
+        {
+            const int d = threadIdx.x;
+            uint32_t run = 0;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                const uint32_t c = counters[w][d];
+                counters[w][d] = run;
+                run += c;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int rd = 0; rd < kRounds; ++rd) {
+            const uint32_t e = first + rd * 32 + lane;
+            if (e < k) {
+                const uint32_t dd = 255u - ((key[rd] >> shift) & 0xFFu);
+                const uint32_t pos = base_s[dd] + counters[warp][dd] + rank[rd];
+                idx_out[pos] = idx[rd];
+                if (LAST) {
+                    if (out_vals) out_vals[pos] = losses[idx[rd]];
+                } else {
+                    keys_out[pos] = key[rd];
+                    atomicAdd(&next_hist[(pos / kTile) * kSortBins + (255u - ((key[rd] >> (shift + 8)) & 0xFFu))], 1u);
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// Small pools: one CTA sorts all N composite keys (key, ~index) in shared memory
+// with a bitonic network; the first k are the selection in loss-descending order.
+constexpr int kSmallThreads = 1024;
+
+__global__ void __launch_bounds__(kSmallThreads)
+small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int32_t* __restrict__ out_idx,
+                  float* __restrict__ out_vals) {
+    __shared__ unsigned long long ck[kSmallN];
+    __shared__ uint32_t warp_tot[kSmallThreads / 32];
+    int n2 = 1;
+    while (n2 < n) n2 <<= 1;
+    for (int i = threadIdx.x; i < n2; i += kSmallThreads)
+        ck[i] = i < n ? (static_cast<unsigned long long>(loss_key(losses[i])) << 32) | (0xFFFFFFFFu - static_cast<uint32_t>(i))
+                      : 0ull;
+    __syncthreads();
+    for (int size = 2; size <= n2; size <<= 1)
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            for (int t = threadIdx.x; t < (n2 >> 1); t += kSmallThreads) {
+                const int lo = ((t / stride) * stride << 1) + (t % stride);
+                const int hi = lo + stride;
+                const bool desc = ((lo & size) == 0);  // this half of the network sorts descending
+                const unsigned long long a = ck[lo], b = ck[hi];
+                if ((a < b) == desc) {
+                    ck[lo] = b;
+                    ck[hi] = a;
+                }
+            }
+            __syncthreads();
+        }
+    if (order == LSGD_ORDER_LOSS_DESC) {
+        for (int j = threadIdx.x; j < k; j += kSmallThreads) {
+            const int32_t i = static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(ck[j]));
+            out_idx[j] = i;
+            if (out_vals) out_vals[j] = losses[i];
+        }
+        return;
+    }
+    // index-ascending: an entry is selected iff its composite key is >= the k-th largest
+    const unsigned long long cut = ck[k - 1];
+    constexpr int kPer = kSmallN / kSmallThreads;  // 4 consecutive indices per thread
+    const int base = threadIdx.x * kPer;
+    bool sel[kPer];
+    uint32_t mine = 0;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+        const int j = base + i;
+        sel[i] = j < n && ((static_cast<unsigned long long>(loss_key(losses[j])) << 32) | (0xFFFFFFFFu - static_cast<uint32_t>(j))) >= cut;
+        mine += sel[i];
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += v;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    uint32_t pos = inc - mine;
+    for (int w = 0; w < warp; ++w) pos += warp_tot[w];
+#pragma unroll
+    for (int i = 0; i < kPer; ++i)
+        if (sel[i]) {
+            out_idx[pos] = base + i;
+            if (out_vals) out_vals[pos] = losses[base + i];
+            ++pos;
+        }
+}
+
+}  // namespace
+
+cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order order, int32_t* out_idx,
+                        float* out_vals, const TopkWorkspace& ws, bool hist0_ready, cudaStream_t s) {
+    if (N <= kSmallN) {
+        small_topk_kernel<<<1, kSmallThreads, 0, s>>>(losses, static_cast<int>(N), static_cast<int>(k),
+                                                      static_cast<int>(order), out_idx, out_vals);
+        return cudaGetLastError();
+    }
+    const int64_t tiles_n = (N + kTile - 1) / kTile;
+    const int grid_n = static_cast<int>(std::min<int64_t>(tiles_n, static_cast<int64_t>(sm_count()) * 8));
+    const uint32_t kk = static_cast<uint32_t>(k);
+    for (int pass = hist0_ready ? 1 : 0; pass < kSelPasses; ++pass)
+        select_hist_kernel<<<grid_n, kThreads, 0, s>>>(losses, N, kk, pass, ws.hist);
+    select_count_kernel<<<grid_n, kThreads, 0, s>>>(losses, N, kk, ws.hist, ws.tile_counts);
+    if (order == LSGD_ORDER_INDEX_ASC) {
+        select_emit_kernel<true><<<grid_n, kThreads, 0, s>>>(losses, N, kk, ws.hist, ws.tile_counts, out_idx, out_vals,
+                                                             nullptr, nullptr);
+        return cudaGetLastError();
+    }
+    const int64_t tiles_k = (k + kTile - 1) / kTile;
+    const size_t th = static_cast<size_t>(tiles_k) * kSortBins;
+    select_emit_kernel<false><<<grid_n, kThreads, 0, s>>>(losses, N, kk, ws.hist, ws.tile_counts, ws.idx[0], nullptr,
+                                                          ws.keys[0], ws.tile_hist);
+    const int grid_k = static_cast<int>(std::min<int64_t>(tiles_k, static_cast<int64_t>(sm_count()) * 4));
+    for (int pass = 0; pass < 3; ++pass)
+        sort_scatter_kernel<false><<<grid_k, kThreads, 0, s>>>(ws.keys[pass & 1], ws.idx[pass & 1], kk, pass,
+                                                               ws.tile_hist + pass * th, ws.keys[(pass + 1) & 1],
+                                                               ws.idx[(pass + 1) & 1], ws.tile_hist + (pass + 1) * th,
+                                                               nullptr, nullptr);
+    sort_scatter_kernel<true><<<grid_k, kThreads, 0, s>>>(ws.keys[1], ws.idx[1], kk, 3, ws.tile_hist + 3 * th, nullptr,
+                                                          out_idx, nullptr, losses, out_vals);
+    return cudaGetLastError();
+}
+
+}  // namespace lsgd

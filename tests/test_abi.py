@@ -1,0 +1,106 @@
+"""The C-ABI library loads and exports what include/lsgd.h declares; host-side
+argument checks and host-only entry points work without a GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    from paper_2508_08540_b200 import build
+
+    build.build_library()
+    from paper_2508_08540_b200 import lsgd
+
+    return lsgd
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "lsgd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"LSGD_API\s+[\w\s\*]+?\b(lsgd_\w+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(L):
+    names = declared_symbols()
+    assert set(names) == set(L.EXPORTS) and len(names) == 11
+    lib = ctypes.CDLL(L.LIB_PATH)
+    for n in names:
+        assert getattr(lib, n) is not None
+
+
+def test_status_strings_and_version(L):
+    assert L.version() >= 100
+    seen = {L.status_string(s) for s in range(7)}
+    assert len(seen) == 7 and L.status_string(0) == "ok"
+    assert L.status_string(99) == "unknown status"
+
+
+def test_workspace_queries(L):
+    assert L.score_workspace_bytes(1000, 1, 10) == 256
+    assert L.score_workspace_bytes(1024, 128, 30522) >= 256 + 4 * 1024 * 128
+    assert L.score_workspace_bytes(-1, 1, 10) == 0 and L.score_workspace_bytes(5, 0, 10) == 0
+    assert L.topk_workspace_bytes(10, 11) == 0 and L.topk_workspace_bytes(-1, 0) == 0
+    a = L.topk_workspace_bytes(1_281_167, 320_000)
+    assert a >= 4 * 4 * 320_000 and a % 256 == 0
+    assert L.score_topk_workspace_bytes(1024, 128, 30522, 256) == L.topk_workspace_bytes(1024, 256) + 4 * 1024 * 128
+    # monotone in k and N
+    assert L.topk_workspace_bytes(50_000, 12_500) <= L.topk_workspace_bytes(50_000, 50_000)
+
+
+def test_weights_from_steps_host_only(L):
+    w = L.weights_from_steps([32] * 8 + [1] * 2)  # Section 5.1 setting: tau_F = 32, tau_S = 1
+    import numpy as np
+
+    assert np.float32(w[0]) == np.float32(32 / 258) and np.float32(w[9]) == np.float32(1 / 258)
+    assert abs(sum(w) - 1.0) < 1e-6
+    with pytest.raises(L.LsgdError) as e:
+        L.weights_from_steps([0, 0, 0])
+    assert e.value.status == L.ERR_INVALID_ARG
+    with pytest.raises(L.LsgdError):
+        L.weights_from_steps([3, -1])
+
+
+def test_argument_errors_are_found_before_any_cuda_call(L):
+    lib = L.lib()
+    one = ctypes.c_float(1.0)
+    ptr = ctypes.c_void_p(0x1000)
+    arr = (ctypes.c_void_p * 1)(0x1000)
+    arrp = ctypes.cast(arr, ctypes.c_void_p)
+    wp = ctypes.cast(ctypes.pointer(one), ctypes.c_void_p)
+    # replica count out of range, NULLs, negative size
+    assert lib.lsgd_aggregate(arrp, wp, 0, 16, ptr, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_aggregate(arrp, wp, 65, 16, ptr, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_aggregate(None, wp, 1, 16, ptr, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_aggregate(arrp, wp, 1, -1, ptr, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_aggregate(arrp, wp, 1, 0, None, None) == L.OK
+    # partial overlap of out with a replica; misaligned replica
+    assert lib.lsgd_aggregate(arrp, wp, 1, 16, ctypes.c_void_p(0x1010), None) == L.ERR_INVALID_ARG
+    bad = (ctypes.c_void_p * 1)(0x1002)
+    assert lib.lsgd_aggregate(ctypes.cast(bad, ctypes.c_void_p), wp, 1, 16, ctypes.c_void_p(0x9000), None) == L.ERR_ALIGNMENT
+    # selector
+    assert lib.lsgd_topk_select(ptr, 10, 11, 0, ptr, None, ptr, 1 << 20, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_topk_select(ptr, 10, -1, 0, ptr, None, ptr, 1 << 20, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_topk_select(ptr, 10, 5, 7, ptr, None, ptr, 1 << 20, None) == L.ERR_UNSUPPORTED
+    assert lib.lsgd_topk_select(ptr, 1 << 31, 5, 0, ptr, None, ptr, 1 << 20, None) == L.ERR_UNSUPPORTED
+    assert lib.lsgd_topk_select(ptr, 10, 0, 0, None, None, None, 0, None) == L.OK
+    assert lib.lsgd_topk_select(None, 10, 5, 0, ptr, None, ptr, 1 << 20, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_topk_select(ptr, 10, 5, 0, ptr, None, ctypes.c_void_p(0x2000), 16, None) == L.ERR_WORKSPACE
+    assert lib.lsgd_topk_select(ptr, 10, 5, 0, ptr, None, ctypes.c_void_p(0x2010), 1 << 20, None) == L.ERR_ALIGNMENT
+    assert lib.lsgd_topk_select(ctypes.c_void_p(0x1001), 10, 5, 0, ptr, None, ptr, 1 << 20, None) == L.ERR_ALIGNMENT
+    # scorer
+    big = ctypes.c_void_p(0x100000)
+    assert lib.lsgd_score_losses(ptr, 5, ptr, 4, 1, 10, -100, big, ptr, 1 << 20, None) == L.ERR_UNSUPPORTED
+    assert lib.lsgd_score_losses(ptr, 0, ptr, 4, 0, 10, -100, big, ptr, 1 << 20, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_score_losses(ptr, 0, ptr, 4, 1, 0, -100, big, ptr, 1 << 20, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_score_losses(ptr, 0, None, 4, 1, 10, -100, big, ptr, 1 << 20, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_score_losses(ptr, 0, ptr, 0, 1, 10, -100, None, None, 0, None) == L.OK
+    assert lib.lsgd_score_losses(ptr, 0, ptr, 4, 1, 10, -100, ctypes.c_void_p(0x1008), ptr, 1 << 20, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_score_losses(ctypes.c_void_p(0x1002), 0, ptr, 4, 1, 10, -100, big, ptr, 1 << 20, None) == L.ERR_ALIGNMENT
+    assert lib.lsgd_score_losses(ptr, 0, ptr, 4, 1, 10, -100, big, ptr, 16, None) == L.ERR_WORKSPACE
+    assert lib.lsgd_score_topk(ptr, 0, ptr, 4, 1, 10, -100, 5, 0, big, ptr, None, ptr, 1 << 20, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_read_device_status(None, None, None) == L.ERR_INVALID_ARG
