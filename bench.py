@@ -317,15 +317,17 @@ def run_gpu(args, cfg):
         h_vals.copy_(vals, non_blocking=True)
         h_out.copy_(out, non_blocking=True)
 
-    step_e2e()
-    barrier()
-    s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    s2.record()
-    for _ in range(e2e_steps):
+    e2e_ms = float("nan")
+    if not args.no_e2e:
         step_e2e()
-    e2.record()
-    barrier()
-    e2e_ms = s2.elapsed_time(e2)
+        barrier()
+        s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s2.record()
+        for _ in range(e2e_steps):
+            step_e2e()
+        e2.record()
+        barrier()
+        e2e_ms = s2.elapsed_time(e2)
 
     t = torch.tensor([total_ms, float(st_ms.sum()), float(ag_ms.sum()), e2e_ms], dtype=torch.float64, device=dev)
     if world > 1:
@@ -388,8 +390,14 @@ def main():
     ap.add_argument("--config", type=int, default=4, choices=sorted(wl.CONFIGS))
     ap.add_argument("--impl", default="lsgd", choices=["lsgd", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--n-samples", type=int, default=0, help="profiling: shrink the pool to this many samples")
+    ap.add_argument("--d-params", type=int, default=0, help="profiling: shrink each replica to this many parameters")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.config]
+    if args.n_samples or args.d_params:
+        n = args.n_samples or cfg.N
+        cfg = wl.scaled(cfg, name=cfg.name + "-scaled", N=n, k=max(1, cfg.k * n // cfg.N), D=args.d_params or cfg.D)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
