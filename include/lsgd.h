@@ -126,6 +126,33 @@ LSGD_API lsgd_status lsgd_topk_select(const float* losses, int64_t N, int64_t k,
                                       void* cuda_stream);
 
 /*
+ * lsgd_topk_select_static — lsgd_topk_select without a workspace argument, for
+ * callers that cannot allocate device memory: code on a path where cudaMalloc
+ * is not allowed (it synchronises the device and can fail late), programs whose
+ * device memory is all owned by another framework's pool, or hosts with no
+ * device allocator of their own.  The paper has no counterpart to this entry
+ * point; it is a convenience of this library.
+ *
+ * The scratch is a fixed array of about 4.3 MiB inside the library's device
+ * image (every GPU that loads the library holds it until the process ends), so
+ * the pool is limited to N <= LSGD_STATIC_TOPK_MAX_N; a larger N returns
+ * LSGD_ERR_UNSUPPORTED and nothing is launched.  Arguments, result and order are
+ * exactly those of lsgd_topk_select.  The call allocates and frees nothing.
+ *
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current).  Make that first call
+ *     outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous
+ *     call's contents; the call clears what has to start at zero.  Two calls that
+ *     can overlap on the GPU (different streams without an ordering between
+ *     them) race on it: keep calls to this entry point on one stream, or order
+ *     them with events.  lsgd_read_device_status does not apply to it.
+ */
+#define LSGD_STATIC_TOPK_MAX_N 262144
+LSGD_API lsgd_status lsgd_topk_select_static(const float* losses, int64_t N, int64_t k, lsgd_order order,
+                                             int32_t* out_idx, float* out_vals, void* cuda_stream);
+
+/*
  * lsgd_score_topk — lsgd_score_losses followed by lsgd_topk_select on its
  * result, enqueued as one sequence in which the scorer's epilogue already
  * builds the selector's first radix histogram.  `losses` ([N], device) is

@@ -25,8 +25,9 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ER
 EXPORTS = (
     "lsgd_version", "lsgd_status_string", "lsgd_score_workspace_bytes", "lsgd_topk_workspace_bytes",
     "lsgd_score_topk_workspace_bytes", "lsgd_score_losses", "lsgd_topk_select", "lsgd_score_topk",
-    "lsgd_aggregate", "lsgd_weights_from_steps", "lsgd_read_device_status",
+    "lsgd_aggregate", "lsgd_weights_from_steps", "lsgd_read_device_status", "lsgd_topk_select_static",
 )
+STATIC_TOPK_MAX_N = 262144
 
 
 class LsgdError(RuntimeError):
@@ -55,6 +56,8 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).argtypes = args
         L.lsgd_score_losses.argtypes = [vp, ci, vp, i64, i64, i64, i64, vp, vp, sz, vp]
         L.lsgd_topk_select.argtypes = [vp, i64, i64, ci, vp, vp, vp, sz, vp]
+        L.lsgd_topk_select_static.argtypes = [vp, i64, i64, ci, vp, vp, vp]
+        L.lsgd_topk_select_static.restype = ci
         L.lsgd_score_topk.argtypes = [vp, ci, vp, i64, i64, i64, i64, i64, ci, vp, vp, vp, vp, sz, vp]
         L.lsgd_aggregate.argtypes = [vp, vp, i32, i64, vp, vp]
         L.lsgd_weights_from_steps.argtypes = [vp, i32, vp]
@@ -151,6 +154,18 @@ def topk_select(losses, k: int, order: int = ORDER_LOSS_DESC, out_idx=None, out_
         ws = workspace(topk_workspace_bytes(N, k), losses.device)
     st = lib().lsgd_topk_select(_p(losses), N, k, order, _p(out_idx), _p(out_vals), _p(ws), ws.numel(), _stream())
     _check("lsgd_topk_select", st)
+    return out_idx, out_vals
+
+
+def topk_select_static(losses, k: int, out_idx, out_vals=None, order: int = ORDER_LOSS_DESC):
+    """lsgd_topk_select_static: the selector on the library's built-in scratch array.
+
+    For callers that must not allocate: the outputs are passed in, no workspace
+    exists, and nothing is allocated here either.  N <= STATIC_TOPK_MAX_N.
+    Calls share one scratch array per device: keep them on one stream.
+    """
+    st = lib().lsgd_topk_select_static(_p(losses), losses.numel(), k, order, _p(out_idx), _p(out_vals), _stream())
+    _check("lsgd_topk_select_static", st)
     return out_idx, out_vals
 
 

@@ -27,7 +27,7 @@ def declared_symbols():
 
 def test_every_declared_symbol_is_exported(L):
     names = declared_symbols()
-    assert set(names) == set(L.EXPORTS) and len(names) == 11
+    assert set(names) == set(L.EXPORTS) and len(names) == 12
     lib = ctypes.CDLL(L.LIB_PATH)
     for n in names:
         assert getattr(lib, n) is not None
