@@ -16,8 +16,9 @@
 // Three row shapes, three kernels (all bound by the bytes of the logits):
 //   tiny rows   (C <= 32)         one thread per row out of a shared-memory tile
 //   short rows  (<= 4064 bytes)   one warp per row, the row held in registers
-//   long rows   (<= ~200 KB)      one CTA per row, the row brought into shared
-//                                 memory by bulk asynchronous copies (TMA, 1-D)
+//   long rows   (<= 256 KB)       a ring of 4 KB chunk buffers per SM filled by bulk
+//                                 asynchronous copies (TMA, 1-D); free-running warps
+//                                 reduce chunks to (max, sum) records
 //   anything longer               one CTA per row, two passes over global memory
 // Rows whose label is ignore_index are never read.
 #include <cuda_bf16.h>
@@ -238,20 +239,49 @@ score_warp_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
 }
 
 // ---------------------------------------------------------------------------
-// Long rows: one CTA per row, the row resident in shared memory.
+// Long rows: a persistent CTA per SM streams rows through a ring of 4 KB chunk
+// buffers in shared memory.
+//   warp 0      producer: takes rows from a device-wide ticket (a batch at a time,
+//               the next batch requested ahead), skips ignored rows, cuts each row
+//               into chunks of 256 vectors and fills the ring with 1-D bulk
+//               asynchronous copies (TMA), tens of chunks ahead of use;
+//   warps 1..   consumers: each takes the next chunk, whichever row it belongs to,
+//               moves it into registers, hands the buffer straight back, and reduces
+//               it to one record (M_c, S_c): the chunk's maximum and its sum of
+//               exp(x - M_c).  Chunks are independent, so warps never wait for each
+//               other and drift apart freely: the special-function unit, which
+//               bounds bf16 rows (one ex2 per 2 bytes), always has warps to serve.
+// The warp that delivers a row's last record combines the records in a fixed
+// order: m = max_c M_c, s = sum_c S_c exp(M_c - m), l = (m - x_y) + log s.
+// If s < 1.5 (a confident row, where log s would lose the small terms next to the 1
+// of the maximum), that warp re-reads the row (an L2 hit as a rule) and sums it with
+// the maximum left out: l = (m - x_y) + log1p(s').
+// The 16-byte-aligned superset of a row is copied and the neighbours' values in
+// its first and last vector are masked in registers; only the first row's head and
+// the last row's tail, which would reach outside the pool, are read element by
+// element.  No CTA-wide barrier exists; every mbarrier wait is bounded.
 // ---------------------------------------------------------------------------
-constexpr int kCtaThreads = 256;
-constexpr int kCtaWarps = kCtaThreads / 32;
-constexpr uint32_t kBulkChunk = 16384;  // bytes per bulk copy
+constexpr int kRingMaxStages = 48;       // 4 KB each
+constexpr int kChunkVecs = 256;          // vectors per chunk: 8 per lane
+constexpr int kChunkBytes = kChunkVecs * 16;
+constexpr int kVecPerLane = kChunkVecs / 32;
+constexpr int kRingBatch = 8;            // rows taken per ticket
+constexpr int kRowSlots = 128;           // rows between their first chunk and their loss (<= stages + warps live at once)
+constexpr int kRecSlots = 256;           // chunk records, by chunk sequence number
+constexpr int kMaxRecsPerRow = 64;       // longer rows (> 256 KB) take the plain kernel
+constexpr int kExpWarps = 24;            // consumer warps
+constexpr int kRingThreads = 32 * (1 + kExpWarps);
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
@@ -278,179 +308,382 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                  "l"(src), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
-__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-struct CtaShared {
-    uint64_t bar;
-    int64_t row;      // row being processed, -1 = no more rows
-    int32_t arg_pos;  // element position of the excluded maximum
-    int32_t give_up;
-    float red_f[kCtaWarps];
-    int32_t red_i[kCtaWarps];
-    float bcast;
+struct RowSlot {
+    int64_t row;
+    int64_t label;
+    int32_t first_rec;  // sequence number of the row's first chunk record
+    int32_t nrec;       // chunks of the row
+    int32_t count;      // records delivered so far
+    float xy;           // the true-class logit (set by the warp whose chunk holds it)
+};
+struct RingShared {
+    uint64_t full[kRingMaxStages];   // the chunk's bytes have landed (producer + TMA)
+    uint64_t empty[kRingMaxStages];  // the buffer may be refilled (the warp that took the chunk)
+    int32_t c_slot[kRingMaxStages];  // per stage: row slot of the chunk, -1 = stop
+    int32_t c_v0[kRingMaxStages];    // first vector of the chunk within its row
+    int32_t c_nv[kRingMaxStages];    // vectors in the chunk
+    int32_t c_rec[kRingMaxStages];   // record sequence number
+    RowSlot rows[kRowSlots];
+    float rec_max[kRecSlots];
+    float rec_sum[kRecSlots];
+    uint32_t next_chunk;             // chunk sequence number handed to the next free warp
+    int32_t abort;                   // a bounded wait ran out somewhere in this CTA
+};
+constexpr int kRingHeaderBytes = 8192;
+static_assert(sizeof(RingShared) <= kRingHeaderBytes, "ring header");
+
+// One element of a row as the raw bits of its type, -inf where j falls outside [0, C).
+template <typename T>
+__device__ __forceinline__ uint32_t ragged_bits(const T* __restrict__ logits, int64_t row, int C, int j) {
+    if constexpr (sizeof(T) == 4) {
+        return (j >= 0 && j < C) ? __float_as_uint(logits[row * C + j]) : 0xFF800000u;
+    } else {
+        return (j >= 0 && j < C) ? static_cast<uint32_t>(__bfloat16_as_ushort(logits[row * C + j])) : 0xFF80u;
+    }
+}
+// One 16-byte vector of a row assembled from global memory element by element:
+// elements j0 .. j0 + EPV - 1 of `row`.
+template <typename T>
+__device__ __forceinline__ uint4 ragged_vector(const T* __restrict__ logits, int64_t row, int C, int j0) {
+    uint4 q;
+    if constexpr (sizeof(T) == 4) {
+        q.x = ragged_bits(logits, row, C, j0);
+        q.y = ragged_bits(logits, row, C, j0 + 1);
+        q.z = ragged_bits(logits, row, C, j0 + 2);
+        q.w = ragged_bits(logits, row, C, j0 + 3);
+    } else {
+        q.x = ragged_bits(logits, row, C, j0) | (ragged_bits(logits, row, C, j0 + 1) << 16);
+        q.y = ragged_bits(logits, row, C, j0 + 2) | (ragged_bits(logits, row, C, j0 + 3) << 16);
+        q.z = ragged_bits(logits, row, C, j0 + 4) | (ragged_bits(logits, row, C, j0 + 5) << 16);
+        q.w = ragged_bits(logits, row, C, j0 + 6) | (ragged_bits(logits, row, C, j0 + 7) << 16);
+    }
+    return q;
+}
+
+// A vector with the element slots outside [lo, hi) replaced by -inf.
+template <typename T>
+__device__ __forceinline__ uint4 mask_outside(uint4 q, int lo, int hi) {
+    uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if constexpr (sizeof(T) == 4) {
+            if (i < lo || i >= hi) w[i] = 0xFF800000u;
+        } else {
+            if (2 * i < lo || 2 * i >= hi) w[i] = (w[i] & 0xFFFF0000u) | 0xFF80u;
+            if (2 * i + 1 < lo || 2 * i + 1 >= hi) w[i] = (w[i] & 0x0000FFFFu) | 0xFF800000u;
+        }
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Running maximum over vectors: packed bf16 pairs for bf16 rows (exact: a maximum rounds nothing).
+template <typename T>
+struct VecMax;
+template <>
+struct VecMax<float> {
+    float m;
+    __device__ VecMax() : m(neg_inf()) {}
+    __device__ void add(const uint4& q) {
+        m = fmaxf(fmaxf(m, fmaxf(__uint_as_float(q.x), __uint_as_float(q.y))),
+                  fmaxf(__uint_as_float(q.z), __uint_as_float(q.w)));
+    }
+    __device__ float get() const { return m; }
+};
+template <>
+struct VecMax<__nv_bfloat16> {
+    __nv_bfloat162 m;
+    __device__ VecMax() : m(__halves2bfloat162(__ushort_as_bfloat16(0xFF80u), __ushort_as_bfloat16(0xFF80u))) {}
+    __device__ void add(const uint4& q) {
+        const __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&q.x),
+                                         *reinterpret_cast<const __nv_bfloat162*>(&q.y));
+        const __nv_bfloat162 b = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&q.z),
+                                         *reinterpret_cast<const __nv_bfloat162*>(&q.w));
+        m = __hmax2(m, __hmax2(a, b));
+    }
+    __device__ float get() const { return fmaxf(__low2float(m), __high2float(m)); }
 };
 
+// The two fp32 values a 32-bit word of the row holds (one for fp32 rows).
 template <typename T>
-__global__ void __launch_bounds__(kCtaThreads)
-score_cta_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
-                      int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0) {
+__device__ __forceinline__ float word_lo(uint32_t w) {
+    return sizeof(T) == 4 ? __uint_as_float(w) : __uint_as_float(w << 16);
+}
+__device__ __forceinline__ float word_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// Packed pairs of fp32 (Blackwell's two-wide fp32 FMA and add).
+struct F2 {
+    unsigned long long v;
+};
+__device__ __forceinline__ F2 pack2(float lo, float hi) {
+    F2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r.v) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(F2 a, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a.v));
+}
+__device__ __forceinline__ F2 fma2(F2 a, F2 b, F2 c) {
+    F2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r.v) : "l"(a.v), "l"(b.v), "l"(c.v));
+    return r;
+}
+__device__ __forceinline__ F2 add2(F2 a, F2 b) {
+    F2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v));
+    return r;
+}
+
+// acc += 2^d exp(x - m) for a pair of elements: one two-wide FMA, two ex2, one two-wide add.
+__device__ __forceinline__ void pair_sum_exp(float x0, float x1, F2 l2e, F2 nml, F2& acc) {
+    float t0, t1;
+    unpack2(fma2(pack2(x0, x1), l2e, nml), t0, t1);
+    acc = add2(acc, pack2(ex2(t0), ex2(t1)));
+}
+
+// a0, a1 += 2^d exp(x - m) over the elements of one vector, in a fixed order.
+template <typename T>
+__device__ __forceinline__ void vec_sum_exp(const uint4& q, F2 l2e, F2 nml, F2& a0, F2& a1) {
+    if constexpr (sizeof(T) == 4) {
+        pair_sum_exp(__uint_as_float(q.x), __uint_as_float(q.y), l2e, nml, a0);
+        pair_sum_exp(__uint_as_float(q.z), __uint_as_float(q.w), l2e, nml, a1);
+    } else {
+        pair_sum_exp(word_lo<T>(q.x), word_hi(q.x), l2e, nml, a0);
+        pair_sum_exp(word_lo<T>(q.y), word_hi(q.y), l2e, nml, a1);
+        pair_sum_exp(word_lo<T>(q.z), word_hi(q.z), l2e, nml, a0);
+        pair_sum_exp(word_lo<T>(q.w), word_hi(q.w), l2e, nml, a1);
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kRingThreads, 1)
+score_ring_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
+                       int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0) {
     constexpr int EPV = Elem<T>::kPerVec;
+    constexpr int kStages = kRingMaxStages;
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    CtaShared& sh = *reinterpret_cast<CtaShared*>(smem_raw);
-    uint32_t* hist_s = reinterpret_cast<uint32_t*>(smem_raw + 128);
-    unsigned char* buf = smem_raw + 128 + (hist0 ? kSelBins * sizeof(uint32_t) : 0);  // 128-byte aligned
+    RingShared& sh = *reinterpret_cast<RingShared*>(smem_raw);
+    uint32_t* hist_s = reinterpret_cast<uint32_t*>(smem_raw + kRingHeaderBytes);
+    unsigned char* bufs = smem_raw + kRingHeaderBytes + (hist0 ? kSelBins * sizeof(uint32_t) : 0);
     Hist0 h{hist_s, hist0};
     h.clear();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t row_bytes = static_cast<int64_t>(C) * sizeof(T);
     if (tid == 0) {
-        mbar_init(&sh.bar, 1);
-        sh.give_up = 0;
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&sh.full[s], 1);
+            mbar_init(&sh.empty[s], 1);
+        }
+        sh.next_chunk = 0;
+        sh.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    uint32_t parity = 0;
 
-    for (;;) {
-        // -- next row: a device-wide ticket, so that CTAs stay busy whatever the mask looks like
-        if (tid == 0) {
-            int64_t r;
-            for (;;) {
-                r = static_cast<int64_t>(atomicAdd(&status->row_ticket, 1u));
-                if (r >= rows) {
-                    r = -1;
-                    break;
-                }
-                const int cls = label_class(labels[r], C, ignore_index);
-                if (cls == 0) break;
-                float l = 0.f;
-                if (cls == 2) {
-                    l = __uint_as_float(0x7FC00000u);
-                    atomicAdd(&status->bad_labels, 1);
-                }
-                row_loss[r] = l;
-                h.add(l);
+    if (warp == 0) {
+        // ---------------- producer ----------------
+        // The whole warp works in step: lane k pushes chunks k, k + 32, ... of the current row, so a
+        // row's copies are issued side by side; the per-row bookkeeping is lane 0's.
+        uint32_t seq = 0;      // chunk sequence number of the row's first chunk (= its record number)
+        uint32_t row_seq = 0;  // rows pushed so far
+        bool failed = false;
+        // claims the stage of chunk sequence number q; false once a wait has run out
+        auto claim = [&](uint32_t q) -> bool {
+            if (failed || sh.abort) return false;
+            if (!mbar_wait(&sh.empty[q % kStages], ((q / kStages) & 1) ^ 1)) {
+                atomicExch(&status->timeout, 1);
+                sh.abort = 1;
+                failed = true;
             }
-            sh.row = r;
-            sh.arg_pos = 0x7FFFFFFF;
-        }
-        __syncthreads();  // also: every thread is done with the previous row's buffer
-        const int64_t row = sh.row;
-        if (row < 0 || sh.give_up) break;
-
-        const uintptr_t ga = reinterpret_cast<uintptr_t>(logits) + row * row_bytes;
-        const int head = static_cast<int>(ga & 15);
-        const int nvec = static_cast<int>((head + row_bytes + 15) >> 4);
-        const int first_body = head ? 1 : 0;                                   // vectors fully inside the row
-        const int end_body = static_cast<int>((head + row_bytes) >> 4);
-        if (tid == 0) {
-            fence_async_proxy();  // earlier generic-proxy accesses of the buffer before the async writes
-            const uint32_t body = static_cast<uint32_t>(end_body - first_body) << 4;
-            mbar_expect_tx(&sh.bar, body);
-            const unsigned char* src = reinterpret_cast<const unsigned char*>(ga - head) + (first_body << 4);
-            unsigned char* dst = buf + (first_body << 4);
-            for (uint32_t o = 0; o < body; o += kBulkChunk)
-                bulk_g2s(dst + o, src + o, min(kBulkChunk, body - o), &sh.bar);
-        } else if (tid >= 32 && tid < 32 + 2 * EPV) {
-            // ragged head and tail: element loads, -inf outside the row
-            const int slot = (tid - 32) % EPV;
-            const bool tail = (tid - 32) >= EPV;
-            const int v = tail ? end_body : 0;
-            if ((tail && end_body < nvec) || (!tail && head)) {
-                const int64_t j = (static_cast<int64_t>(v) * 16 - head) / static_cast<int>(sizeof(T)) + slot;
-                T val = Elem<T>::neg_inf_elem();
-                if (j >= 0 && j < C) val = logits[row * C + j];
-                reinterpret_cast<T*>(buf)[v * EPV + slot] = val;
+            return !failed;
+        };
+        auto push_row = [&](int64_t r, int64_t y) {
+            const uintptr_t ga = reinterpret_cast<uintptr_t>(logits) + r * row_bytes;
+            const int head = static_cast<int>(ga & 15);
+            const int nvec = static_cast<int>((head + row_bytes + 15) >> 4);
+            const int nchunk = (nvec + kChunkVecs - 1) / kChunkVecs;
+            // vectors that would reach outside the pool are not copied
+            const int skip_head = (head && r == 0) ? 1 : 0;
+            const int skip_tail = (((head + row_bytes) & 15) && r == rows - 1) ? 1 : 0;
+            const int slot = row_seq++ % kRowSlots;
+            if (lane == 0) {
+                RowSlot& rs = sh.rows[slot];
+                rs.row = r;
+                rs.label = y;
+                rs.first_rec = static_cast<int32_t>(seq);
+                rs.nrec = nchunk;
+                rs.count = 0;
             }
-        }
-        float xy = 0.f;
-        if (tid == 0) xy = Elem<T>::widen(__ldg(logits + row * C + labels[row]));
-        if (!mbar_wait(&sh.bar, parity)) {
-            // the copy did not land in time: flag it, give it one more bounded wait so that
-            // nothing is still writing into shared memory when the CTA leaves, and stop
-            atomicExch(&status->timeout, 1);
-            mbar_wait(&sh.bar, parity);
-            sh.give_up = 1;
-        }
-        parity ^= 1;
-        __syncthreads();
-        if (sh.give_up) break;
-
-        // -- pass 1: maximum
-        const uint4* vec = reinterpret_cast<const uint4*>(buf);
-        float m;
-        if constexpr (EPV == 4) {
-            m = neg_inf();
-            for (int v = tid; v < nvec; v += kCtaThreads) {
-                const uint4 q = vec[v];
-                m = fmaxf(fmaxf(m, fmaxf(__uint_as_float(q.x), __uint_as_float(q.y))),
-                          fmaxf(__uint_as_float(q.z), __uint_as_float(q.w)));
+            __syncwarp();  // the slot is written before any lane publishes a chunk of the row
+            const unsigned char* src = reinterpret_cast<const unsigned char*>(ga - head);
+            for (int k = lane; k < nchunk; k += 32) {
+                const uint32_t q = seq + k;
+                if (!claim(q)) break;
+                const int s = q % kStages;
+                const int v0 = k * kChunkVecs;
+                const int nv = min(kChunkVecs, nvec - v0);
+                const int cb = (k == 0) ? skip_head : 0;
+                const int ce = nv - ((k == nchunk - 1) ? skip_tail : 0);
+                sh.c_slot[s] = slot;
+                sh.c_v0[s] = v0;
+                sh.c_nv[s] = nv;
+                sh.c_rec[s] = static_cast<int32_t>(q);
+                const uint32_t bytes = static_cast<uint32_t>(max(ce - cb, 0)) << 4;
+                mbar_expect_tx(&sh.full[s], bytes);
+                if (bytes)
+                    bulk_g2s(bufs + static_cast<size_t>(s) * kChunkBytes + (cb << 4),
+                             src + (static_cast<size_t>(v0 + cb) << 4), bytes, &sh.full[s]);
             }
-        } else {
-            __nv_bfloat162 mm = __halves2bfloat162(Elem<T>::neg_inf_elem(), Elem<T>::neg_inf_elem());
-            for (int v = tid; v < nvec; v += kCtaThreads) {
-                const uint4 q = vec[v];
-                const __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&q.x),
-                                                 *reinterpret_cast<const __nv_bfloat162*>(&q.y));
-                const __nv_bfloat162 b = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&q.z),
-                                                 *reinterpret_cast<const __nv_bfloat162*>(&q.w));
-                mm = __hmax2(mm, __hmax2(a, b));
-            }
-            m = fmaxf(__low2float(mm), __high2float(mm));
-        }
-        const float my_max = m;
-        m = warp_max(m);
-        if (lane == 0) sh.red_f[warp] = m;
-        __syncthreads();
-        m = sh.red_f[0];
-#pragma unroll
-        for (int w = 1; w < kCtaWarps; ++w) m = fmaxf(m, sh.red_f[w]);
-
-        // -- take one occurrence of the maximum (the first) out of the row
-        if (my_max == m) {
-            int pos = 0x7FFFFFFF;
-            for (int v = tid; v < nvec && pos == 0x7FFFFFFF; v += kCtaThreads)
-                for (int e = 0; e < EPV; ++e)
-                    if (Elem<T>::widen(reinterpret_cast<const T*>(buf)[v * EPV + e]) == m) {
-                        pos = v * EPV + e;
-                        break;
+            seq += nchunk;
+            __syncwarp();
+        };
+        // lane 0 draws the ticket, lanes 0 .. kRingBatch-1 fetch one label each
+        auto take = [&](int64_t& base, int64_t& lab) {
+            uint32_t t = 0;
+            if (lane == 0) t = atomicAdd(&status->row_ticket, static_cast<uint32_t>(kRingBatch));
+            base = static_cast<int64_t>(__shfl_sync(0xFFFFFFFFu, t, 0));
+            lab = (lane < kRingBatch && base + lane < rows) ? labels[base + lane] : ignore_index;
+        };
+        // the ticket and the labels of the NEXT batch are requested before the current batch is
+        // worked through, so their round trips to memory hide behind the copies being issued
+        int64_t next_base, next_lab;
+        take(next_base, next_lab);
+        for (;;) {
+            const int64_t base = next_base, lab = next_lab;
+            if (base >= rows || __any_sync(0xFFFFFFFFu, failed || sh.abort)) break;
+            take(next_base, next_lab);
+            for (int j = 0; j < kRingBatch && base + j < rows; ++j) {
+                const int64_t r = base + j;
+                const int64_t y = __shfl_sync(0xFFFFFFFFu, lab, j);
+                const int cls = label_class(y, C, ignore_index);
+                if (cls == 0) {
+                    push_row(r, y);
+                } else if (lane == 0) {
+                    float l = 0.f;
+                    if (cls == 2) {
+                        l = __uint_as_float(0x7FC00000u);
+                        atomicAdd(&status->bad_labels, 1);
                     }
-            atomicMin(&sh.arg_pos, pos);
-        }
-        __syncthreads();
-        if (tid == 0) reinterpret_cast<T*>(buf)[sh.arg_pos] = Elem<T>::neg_inf_elem();
-        __syncthreads();
-
-        // -- pass 2: sum of exponentials (everything left is <= m; -inf gives 0)
-        const RowScale rs(m);
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-        for (int v = tid; v < nvec; v += kCtaThreads) {
-            const uint4 q = vec[v];
-            if constexpr (EPV == 4) {
-                s0 += ex2(fmaf(__uint_as_float(q.x), kLog2e, rs.nml));
-                s1 += ex2(fmaf(__uint_as_float(q.y), kLog2e, rs.nml));
-                s2 += ex2(fmaf(__uint_as_float(q.z), kLog2e, rs.nml));
-                s3 += ex2(fmaf(__uint_as_float(q.w), kLog2e, rs.nml));
-            } else {
-                s0 += ex2(fmaf(__uint_as_float(q.x << 16), kLog2e, rs.nml));
-                s1 += ex2(fmaf(__uint_as_float(q.x & 0xFFFF0000u), kLog2e, rs.nml));
-                s2 += ex2(fmaf(__uint_as_float(q.y << 16), kLog2e, rs.nml));
-                s3 += ex2(fmaf(__uint_as_float(q.y & 0xFFFF0000u), kLog2e, rs.nml));
-                s0 += ex2(fmaf(__uint_as_float(q.z << 16), kLog2e, rs.nml));
-                s1 += ex2(fmaf(__uint_as_float(q.z & 0xFFFF0000u), kLog2e, rs.nml));
-                s2 += ex2(fmaf(__uint_as_float(q.w << 16), kLog2e, rs.nml));
-                s3 += ex2(fmaf(__uint_as_float(q.w & 0xFFFF0000u), kLog2e, rs.nml));
+                    row_loss[r] = l;
+                    h.add(l);
+                }
             }
         }
-        float s = warp_sum((s0 + s1) + (s2 + s3));
-        if (lane == 0) sh.red_f[warp] = s;  // the two barriers above separate this from the reads of the maxima
-        __syncthreads();
-        if (tid == 0) {
-            s = sh.red_f[0];
+        // stop markers: every consumer warp takes exactly one
+        if (lane < kExpWarps) {
+            const uint32_t q = seq + lane;
+            claim(q);  // after a failed wait nothing is waited for any more
+            sh.c_slot[q % kStages] = -1;
+            mbar_arrive(&sh.full[q % kStages]);
+        }
+        __syncwarp();
+    } else {
+        // ---------------- consumers ----------------
+        for (;;) {
+            uint32_t c = 0;
+            if (lane == 0) c = atomicAdd(&sh.next_chunk, 1u);
+            c = __shfl_sync(0xFFFFFFFFu, c, 0);
+            const int s = c % kStages;
+            if (!mbar_wait(&sh.full[s], (c / kStages) & 1)) {
+                atomicExch(&status->timeout, 1);
+                sh.abort = 1;
+                mbar_wait(&sh.full[s], (c / kStages) & 1);  // nothing may still be landing when the CTA leaves
+                break;  // no barrier ties this warp to the others: it can simply leave
+            }
+            const int slot = sh.c_slot[s];
+            if (slot < 0) break;
+            RowSlot& rs = sh.rows[slot];
+            const int v0 = sh.c_v0[s], nv = sh.c_nv[s], rec = sh.c_rec[s] % kRecSlots;
+            const int64_t row = rs.row;
+            const uintptr_t ga = reinterpret_cast<uintptr_t>(logits) + row * row_bytes;
+            const int head = static_cast<int>(ga & 15);
+            const int nvec = static_cast<int>((head + row_bytes + 15) >> 4);
+            const int tail = static_cast<int>((head + row_bytes) & 15);  // bytes of the row in its last vector (0 = all 16)
+            const int e0 = -head / static_cast<int>(sizeof(T));          // element index of slot 0 of vector 0
+            const uint4* vec = reinterpret_cast<const uint4*>(bufs + static_cast<size_t>(s) * kChunkBytes);
+
+            // -- the chunk into registers; the two ends of a row need care
+            uint4 raw[kVecPerLane];
+            const uint32_t ninf = EPV == 4 ? 0xFF800000u : 0xFF80FF80u;
+            const int last_i = (tail && v0 + nv == nvec) ? nv - 1 : -1;  // where the row ends inside a vector
 #pragma unroll
-            for (int w = 1; w < kCtaWarps; ++w) s += sh.red_f[w];
-            const float loss = finish_loss(m, xy, s, 1, rs);
-            row_loss[row] = loss;
-            h.add(loss);
+            for (int u = 0; u < kVecPerLane; ++u) {
+                const int i = lane + 32 * u;
+                raw[u] = i < nv ? vec[i] : make_uint4(ninf, ninf, ninf, ninf);
+                if (i == last_i)
+                    raw[u] = row == rows - 1 ? ragged_vector<T>(logits, row, C, e0 + (nvec - 1) * EPV)
+                                             : mask_outside<T>(raw[u], 0, tail / static_cast<int>(sizeof(T)));
+            }
+            if (lane == 0 && v0 == 0 && head)  // the row starts inside its first vector
+                raw[0] = row == 0 ? ragged_vector<T>(logits, row, C, e0) : mask_outside<T>(raw[0], -e0, EPV);
+            {  // the true-class logit, if this chunk holds it
+                const int64_t ey = rs.label - e0;  // element slot within the row's vectors
+                const int vy = static_cast<int>(ey / EPV);
+                if (lane == 0 && vy >= v0 && vy < v0 + nv)
+                    rs.xy = (row == 0 || row == rows - 1) ? Elem<T>::widen(logits[row * C + rs.label])
+                                                          : Elem<T>::widen(reinterpret_cast<const T*>(vec)[ey - static_cast<int64_t>(v0) * EPV]);
+            }
+
+            // -- chunk maximum (every lane's loads have returned once the shuffles are through)
+            VecMax<T> vm;
+#pragma unroll
+            for (int u = 0; u < kVecPerLane; ++u) vm.add(raw[u]);
+            const float M = warp_max(vm.get());
+            if (lane == 0) mbar_arrive(&sh.empty[s]);  // the chunk is in registers: the buffer can be refilled
+
+            // -- chunk sum of exponentials
+            const RowScale sc(M);
+            const F2 l2e = pack2(kLog2e, kLog2e), nml2 = pack2(sc.nml, sc.nml);
+            F2 a0 = pack2(0.f, 0.f), a1 = a0;
+#pragma unroll
+            for (int u = 0; u < kVecPerLane; ++u) vec_sum_exp<T>(raw[u], l2e, nml2, a0, a1);
+            float p0, p1, p2, p3;
+            unpack2(a0, p0, p1);
+            unpack2(a1, p2, p3);
+            const float S = warp_sum((p0 + p1) + (p2 + p3)) * sc.corr;
+
+            // -- record; the warp that delivers the row's last record finishes the row
+            int last = 0;
+            if (lane == 0) {
+                sh.rec_max[rec] = M;
+                sh.rec_sum[rec] = S;
+                __threadfence_block();
+                last = atomicAdd(&rs.count, 1) == rs.nrec - 1;
+            }
+            last = __shfl_sync(0xFFFFFFFFu, last, 0);
+            if (!last) continue;
+            __threadfence_block();
+            const int nrec = rs.nrec, first = rs.first_rec;
+            const int ia = lane, ib = lane + 32;
+            const float Ma = ia < nrec ? sh.rec_max[(first + ia) % kRecSlots] : neg_inf();
+            const float Mb = ib < nrec ? sh.rec_max[(first + ib) % kRecSlots] : neg_inf();
+            const float Sa = ia < nrec ? sh.rec_sum[(first + ia) % kRecSlots] : 0.f;
+            const float Sb = ib < nrec ? sh.rec_sum[(first + ib) % kRecSlots] : 0.f;
+            const float m = warp_max(fmaxf(Ma, Mb));
+            const float ssum = warp_sum(Sa * ex2((Ma - m) * kLog2e) + Sb * ex2((Mb - m) * kLog2e));
+            const float xy = rs.xy;
+            float loss;
+            if (ssum >= 1.5f) {
+                loss = (m - xy) + logf(ssum);
+            } else {
+                // a confident row: the sum again with the maximum left out, from a second read of the row
+                const RowScale fs(m);
+                const T* x = logits + row * C;
+                float s_lt = 0.f;
+                int n_max = 0;
+                for (int j = lane; j < C; j += 32) {
+                    const float v = Elem<T>::widen(x[j]);
+                    if (v < m) s_lt += ex2(fmaf(v, kLog2e, fs.nml));
+                    else ++n_max;
+                }
+                s_lt = warp_sum(s_lt);
+                n_max = warp_sum(n_max);
+                loss = finish_loss(m, xy, s_lt, n_max, fs);
+            }
+            if (lane == 0) {
+                row_loss[row] = loss;
+                h.add(loss);
+            }
         }
     }
     __syncthreads();
@@ -461,6 +694,9 @@ score_cta_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ 
 // Rows too long for shared memory: one CTA per row, two passes over global
 // memory with plain element loads.  A plain fallback, not a tuned path.
 // ---------------------------------------------------------------------------
+constexpr int kCtaThreads = 256;
+constexpr int kCtaWarps = kCtaThreads / 32;
+
 template <typename T>
 __global__ void __launch_bounds__(kCtaThreads)
 score_huge_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int64_t C,
@@ -592,15 +828,16 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
         else go(score_warp_rows_kernel<T, 8>);
         return cudaGetLastError();
     }
-    const size_t smem = 128 + (hist0 ? kSelBins * sizeof(uint32_t) : 0) + static_cast<size_t>((row_bytes + 32 + 127) / 128 * 128);
-    if (smem <= kMaxDynSmem) {
-        cudaError_t e = cudaFuncSetAttribute(score_cta_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (need_vec <= static_cast<int64_t>(kMaxRecsPerRow) * kChunkVecs) {
+        // ring of chunk buffers in shared memory, one persistent CTA per SM
+        const size_t fixed = kRingHeaderBytes + (hist0 ? kSelBins * sizeof(uint32_t) : 0);
+        const size_t smem = fixed + static_cast<size_t>(kRingMaxStages) * kChunkBytes;
+        const int grid = static_cast<int>(std::min<int64_t>(rows, sms));
+        cudaError_t e = cudaFuncSetAttribute(score_ring_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              static_cast<int>(kMaxDynSmem));
         if (e != cudaSuccess) return e;
-        const int bps = blocks_per_sm(score_cta_rows_kernel<T>, kCtaThreads, smem);
-        const int grid = static_cast<int>(std::min<int64_t>(rows, static_cast<int64_t>(sms) * bps));
-        score_cta_rows_kernel<T><<<grid, kCtaThreads, smem, s>>>(logits, labels, rows, static_cast<int>(C),
-                                                                  ignore_index, row_loss, status, hist0);
+        score_ring_rows_kernel<T><<<grid, kRingThreads, smem, s>>>(logits, labels, rows, static_cast<int>(C),
+                                                                   ignore_index, row_loss, status, hist0);
         return cudaGetLastError();
     }
     const int grid = static_cast<int>(std::min<int64_t>(rows, static_cast<int64_t>(sms) * 8));
