@@ -204,6 +204,26 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of `values` over all ranks (identity without a process group).
+
+    Every multi-GPU number is the slowest rank's: ranks run independent replicas of the round,
+    so the job is as fast as its slowest member.
+    """
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_throughput(world: int, units_per_rank: float, steps: int, ms: float) -> float:
+    """Whole-job units per second: every rank processed `units_per_rank` per step, in `ms` (max over ranks)."""
+    return world * units_per_rank * steps / (ms * 1e-3)
+
+
 def workload_config(cfg, residency: str):
     return {
         "workload": f"config {cfg.cfg_id} ({cfg.name}-scale round): pool {cfg.N} x {cfg.T} x {cfg.C} {cfg.dtype} logits, "
@@ -329,10 +349,7 @@ def run_gpu(args, cfg):
         barrier()
         e2e_ms = s2.elapsed_time(e2)
 
-    t = torch.tensor([total_ms, float(st_ms.sum()), float(ag_ms.sum()), e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, st_sum, ag_sum, e2e_ms = t.tolist()
+    total_ms, st_sum, ag_sum, e2e_ms = max_over_ranks([total_ms, float(st_ms.sum()), float(ag_ms.sum()), e2e_ms], dev)
     if rank == 0:
         peak, peak_src = measured_peak()
         st_bytes = score_topk_bytes(cfg, h_labels.numpy())
@@ -341,7 +358,7 @@ def run_gpu(args, cfg):
         ag_gbs = ag_bytes * args.steps / (ag_sum * 1e-3) / 1e9
         n_launch = launches_per_step(cfg)
         line = {
-            "metric": "score+top-k samples/s", "value": world * cfg.N * args.steps / (st_sum * 1e-3), "unit": "samples/s",
+            "metric": "score+top-k samples/s", "value": job_throughput(world, cfg.N, args.steps, st_sum), "unit": "samples/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": workload_config(cfg, "resident in HBM"),
