@@ -153,6 +153,19 @@ __device__ __forceinline__ uint32_t prefix_mask(int pass) { return pass == 0 ? 0
 // Loads the 16 keys thread `threadIdx.x` owns in tile `tile` (consecutive
 // indices), 0 beyond N.  Key 0 belongs to no loss (loss_key never returns it).
 __device__ __forceinline__ void load_keys(const float* __restrict__ losses, int64_t N, int64_t base, uint32_t (&key)[kPerThread]) {
+    if (base + kPerThread <= N && (reinterpret_cast<uintptr_t>(losses + base) & 15) == 0) {
+        float4 q[kPerThread / 4];
+#pragma unroll
+        for (int i = 0; i < kPerThread / 4; ++i) q[i] = reinterpret_cast<const float4*>(losses + base)[i];
+#pragma unroll
+        for (int i = 0; i < kPerThread / 4; ++i) {
+            key[4 * i] = loss_key(q[i].x);
+            key[4 * i + 1] = loss_key(q[i].y);
+            key[4 * i + 2] = loss_key(q[i].z);
+            key[4 * i + 3] = loss_key(q[i].w);
+        }
+        return;
+    }
 #pragma unroll
     for (int i = 0; i < kPerThread; ++i) {
         const int64_t j = base + i;
@@ -174,12 +187,24 @@ select_hist_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, int 
     const uint32_t mask = prefix_mask(pass);
     for (int64_t tile = blockIdx.x; tile * kTile < N; tile += gridDim.x) {
         const int64_t base = tile * kTile;
-#pragma unroll 4
+        float v[kPerThread];
+#pragma unroll
+        for (int i = 0; i < kPerThread; ++i) {  // all loads first: they are independent
+            const int64_t j = base + i * kThreads + threadIdx.x;
+            v[i] = j < N ? losses[j] : 0.f;
+        }
+#pragma unroll
         for (int i = 0; i < kPerThread; ++i) {
             const int64_t j = base + i * kThreads + threadIdx.x;
-            if (j < N) {
-                const uint32_t key = loss_key(losses[j]);
-                if ((key & mask) == prefix) atomicAdd(&hist_s[digit_of(key, pass)], 1u);
+            const uint32_t key = loss_key(v[i]);
+            const bool in = j < N && (key & mask) == prefix;
+            if (pass == 0) {
+                // every key counts and losses crowd into a few bins: one atomic per distinct digit and warp
+                const uint32_t d = in ? digit_of(key, 0) : 0xFFFFFFFFu;
+                const uint32_t peers = __match_any_sync(0xFFFFFFFFu, d);
+                if (in && (threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist_s[d], __popc(peers));
+            } else if (in) {
+                atomicAdd(&hist_s[digit_of(key, pass)], 1u);
             }
         }
     }
@@ -202,14 +227,18 @@ select_count_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, con
         if (threadIdx.x < 2) cnt[threadIdx.x] = 0;
         __syncthreads();
         uint32_t gt = 0, eq = 0;
-#pragma unroll 4
+        float v[kPerThread];
+#pragma unroll
         for (int i = 0; i < kPerThread; ++i) {
             const int64_t j = tile * kTile + i * kThreads + threadIdx.x;
-            if (j < N) {
-                const uint32_t key = loss_key(losses[j]);
-                gt += key > T;
-                eq += key == T;
-            }
+            v[i] = j < N ? losses[j] : 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < kPerThread; ++i) {
+            const int64_t j = tile * kTile + i * kThreads + threadIdx.x;
+            const uint32_t key = j < N ? loss_key(v[i]) : 0u;  // key 0 belongs to no loss and is below every threshold
+            gt += key > T;
+            eq += key == T;
         }
         gt = warp_sum(static_cast<int>(gt));
         eq = warp_sum(static_cast<int>(eq));
@@ -330,11 +359,15 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
         int32_t idx[kRounds];
         const uint32_t first = tile * kTile + warp * (kRounds * 32);
 #pragma unroll
+        for (int rd = 0; rd < kRounds; ++rd) {  // all loads first: they are independent
+            const uint32_t e = first + rd * 32 + lane;
+            key[rd] = e < k ? keys_in[e] : 0u;
+            idx[rd] = e < k ? idx_in[e] : 0;
+        }
+#pragma unroll
         for (int rd = 0; rd < kRounds; ++rd) {
             const uint32_t e = first + rd * 32 + lane;
             const bool live = e < k;
-            key[rd] = live ? keys_in[e] : 0u;
-            idx[rd] = live ? idx_in[e] : 0;
             const uint32_t dd = live ? 255u - ((key[rd] >> shift) & 0xFFu) : 256u;
             const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dd);
             const int leader = __ffs(peers) - 1;
