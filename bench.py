@@ -224,6 +224,15 @@ def job_throughput(world: int, units_per_rank: float, steps: int, ms: float) -> 
     return world * units_per_rank * steps / (ms * 1e-3)
 
 
+# DRAM traffic per launch (dram__bytes_read + dram__bytes_write) from the ncu captures summarised under
+# profiles/, taken on a scaled-down case and scaled to a full launch by the units processed.  Only for the
+# kernels and workloads that were captured; None elsewhere (and to be reset when a kernel changes).
+NCU_TRAFFIC_BYTES = {
+    ("score", 4): 7.26e9,      # profiles/score_ring_rows_bf16_cfg4.md: 907.6 MB for 128 of 1024 sequences
+    ("aggregate", 4): 4.70e9,  # profiles/aggregate_vec4_cfg4.md: 687.0 MB for 16,000,000 of 109,482,240 parameters
+}
+
+
 def workload_config(cfg, residency: str):
     return {
         "workload": f"config {cfg.cfg_id} ({cfg.name}-scale round): pool {cfg.N} x {cfg.T} x {cfg.C} {cfg.dtype} logits, "
@@ -370,10 +379,13 @@ def run_gpu(args, cfg):
                             "algorithmic_bytes": ag_bytes},
             "round_samples_per_s": world * cfg.N * args.steps / (total_ms * 1e-3),
             "roofline": {"bound": "hbm", "kernel": "lsgd_score_topk (scorer kernel + memset, sequence mean, selector)",
-                         "achieved": st_gbs, "peak": peak, "unit": "GB/s", "frac": st_gbs / peak, "traffic": None,
+                         "achieved": st_gbs, "peak": peak, "unit": "GB/s", "frac": st_gbs / peak,
+                         "traffic": NCU_TRAFFIC_BYTES.get(("score", cfg.cfg_id)) if not (args.n_samples or args.d_params) else None,
                          "peak_source": peak_src},
             "roofline_aggregate": {"bound": "hbm", "kernel": "aggregate_vec4_kernel", "achieved": ag_gbs, "peak": peak,
-                                   "unit": "GB/s", "frac": ag_gbs / peak, "traffic": None, "peak_source": peak_src},
+                                   "unit": "GB/s", "frac": ag_gbs / peak,
+                                   "traffic": NCU_TRAFFIC_BYTES.get(("aggregate", cfg.cfg_id)) if not (args.n_samples or args.d_params) else None,
+                                   "peak_source": peak_src},
             "e2e": {"value": world * cfg.N * e2e_steps / (e2e_ms * 1e-3), "unit": "samples/s", "ms_per_step": e2e_ms / e2e_steps,
                     "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "note": "whole step (score+top-k and aggregation) incl. copies; bound by the host link"},
