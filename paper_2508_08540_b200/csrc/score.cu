@@ -256,10 +256,13 @@ score_warp_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
 // If s < 1.5 (a confident row, where log s would lose the small terms next to the 1
 // of the maximum), that warp re-reads the row (an L2 hit as a rule) and sums it with
 // the maximum left out: l = (m - x_y) + log1p(s').
-// The 16-byte-aligned superset of a row is copied and the neighbours' values in
-// its first and last vector are masked in registers; only the first row's head and
-// the last row's tail, which would reach outside the pool, are read element by
-// element.  No CTA-wide barrier exists; every mbarrier wait is bounded.
+// Only the vectors that lie wholly inside a row are bulk-copied, so nothing needs
+// masking in the chunk loop; the (at most two) vectors in which a row starts or ends
+// are read element by element by the warp that finishes the row and enter the
+// combination as records of their own.  Nothing outside a row is ever read.
+// No CTA-wide barrier exists; every mbarrier wait is bounded.  Copies complete out
+// of order, so a stage's barrier can be a whole lap behind the chunk a fast warp is
+// asking for: a stage is taken only when its record number is the chunk's.
 // ---------------------------------------------------------------------------
 constexpr int kRingMaxStages = 48;       // 4 KB each
 constexpr int kChunkVecs = 256;          // vectors per chunk: 8 per lane
@@ -332,50 +335,6 @@ struct RingShared {
 };
 constexpr int kRingHeaderBytes = 8192;
 static_assert(sizeof(RingShared) <= kRingHeaderBytes, "ring header");
-
-// One element of a row as the raw bits of its type, -inf where j falls outside [0, C).
-template <typename T>
-__device__ __forceinline__ uint32_t ragged_bits(const T* __restrict__ logits, int64_t row, int C, int j) {
-    if constexpr (sizeof(T) == 4) {
-        return (j >= 0 && j < C) ? __float_as_uint(logits[row * C + j]) : 0xFF800000u;
-    } else {
-        return (j >= 0 && j < C) ? static_cast<uint32_t>(__bfloat16_as_ushort(logits[row * C + j])) : 0xFF80u;
-    }
-}
-// One 16-byte vector of a row assembled from global memory element by element:
-// elements j0 .. j0 + EPV - 1 of `row`.
-template <typename T>
-__device__ __forceinline__ uint4 ragged_vector(const T* __restrict__ logits, int64_t row, int C, int j0) {
-    uint4 q;
-    if constexpr (sizeof(T) == 4) {
-        q.x = ragged_bits(logits, row, C, j0);
-        q.y = ragged_bits(logits, row, C, j0 + 1);
-        q.z = ragged_bits(logits, row, C, j0 + 2);
-        q.w = ragged_bits(logits, row, C, j0 + 3);
-    } else {
-        q.x = ragged_bits(logits, row, C, j0) | (ragged_bits(logits, row, C, j0 + 1) << 16);
-        q.y = ragged_bits(logits, row, C, j0 + 2) | (ragged_bits(logits, row, C, j0 + 3) << 16);
-        q.z = ragged_bits(logits, row, C, j0 + 4) | (ragged_bits(logits, row, C, j0 + 5) << 16);
-        q.w = ragged_bits(logits, row, C, j0 + 6) | (ragged_bits(logits, row, C, j0 + 7) << 16);
-    }
-    return q;
-}
-
-// A vector with the element slots outside [lo, hi) replaced by -inf.
-template <typename T>
-__device__ __forceinline__ uint4 mask_outside(uint4 q, int lo, int hi) {
-    uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        if constexpr (sizeof(T) == 4) {
-            if (i < lo || i >= hi) w[i] = 0xFF800000u;
-        } else {
-            if (2 * i < lo || 2 * i >= hi) w[i] = (w[i] & 0xFFFF0000u) | 0xFF80u;
-            if (2 * i + 1 < lo || 2 * i + 1 >= hi) w[i] = (w[i] & 0x0000FFFFu) | 0xFF800000u;
-        }
-    }
-    return make_uint4(w[0], w[1], w[2], w[3]);
-}
 
 // Running maximum over vectors: packed bf16 pairs for bf16 rows (exact: a maximum rounds nothing).
 template <typename T>
@@ -501,17 +460,18 @@ score_ring_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
             const uintptr_t ga = reinterpret_cast<uintptr_t>(logits) + r * row_bytes;
             const int head = static_cast<int>(ga & 15);
             const int nvec = static_cast<int>((head + row_bytes + 15) >> 4);
-            const int nchunk = (nvec + kChunkVecs - 1) / kChunkVecs;
-            // vectors that would reach outside the pool are not copied
-            const int skip_head = (head && r == 0) ? 1 : 0;
-            const int skip_tail = (((head + row_bytes) & 15) && r == rows - 1) ? 1 : 0;
+            // only the vectors that lie wholly inside the row travel by bulk copy; the (at most two) vectors in
+            // which the row starts or ends are read element by element by the warp that finishes the row
+            const int first = head ? 1 : 0;
+            const int last = ((head + row_bytes) & 15) ? nvec - 1 : nvec;
+            const int nchunk = (max(last - first, 0) + kChunkVecs - 1) / kChunkVecs;
             const int slot = row_seq++ % kRowSlots;
             if (lane == 0) {
                 RowSlot& rs = sh.rows[slot];
                 rs.row = r;
                 rs.label = y;
                 rs.first_rec = static_cast<int32_t>(seq);
-                rs.nrec = nchunk;
+                rs.nrec = nchunk;  // >= 1: rows of this kernel span hundreds of vectors
                 rs.count = 0;
             }
             __syncwarp();  // the slot is written before any lane publishes a chunk of the row
@@ -520,19 +480,16 @@ score_ring_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
                 const uint32_t q = seq + k;
                 if (!claim(q)) break;
                 const int s = q % kStages;
-                const int v0 = k * kChunkVecs;
-                const int nv = min(kChunkVecs, nvec - v0);
-                const int cb = (k == 0) ? skip_head : 0;
-                const int ce = nv - ((k == nchunk - 1) ? skip_tail : 0);
+                const int v0 = first + k * kChunkVecs;
+                const int nv = min(kChunkVecs, last - v0);
                 sh.c_slot[s] = slot;
                 sh.c_v0[s] = v0;
                 sh.c_nv[s] = nv;
                 sh.c_rec[s] = static_cast<int32_t>(q);
-                const uint32_t bytes = static_cast<uint32_t>(max(ce - cb, 0)) << 4;
+                const uint32_t bytes = static_cast<uint32_t>(nv) << 4;
                 mbar_expect_tx(&sh.full[s], bytes);
-                if (bytes)
-                    bulk_g2s(bufs + static_cast<size_t>(s) * kChunkBytes + (cb << 4),
-                             src + (static_cast<size_t>(v0 + cb) << 4), bytes, &sh.full[s]);
+                bulk_g2s(bufs + static_cast<size_t>(s) * kChunkBytes, src + (static_cast<size_t>(v0) << 4), bytes,
+                         &sh.full[s]);
             }
             seq += nchunk;
             __syncwarp();
@@ -574,6 +531,7 @@ score_ring_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
             const uint32_t q = seq + lane;
             claim(q);  // after a failed wait nothing is waited for any more
             sh.c_slot[q % kStages] = -1;
+            sh.c_rec[q % kStages] = static_cast<int32_t>(q);
             mbar_arrive(&sh.full[q % kStages]);
         }
         __syncwarp();
@@ -584,10 +542,23 @@ score_ring_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
             if (lane == 0) c = atomicAdd(&sh.next_chunk, 1u);
             c = __shfl_sync(0xFFFFFFFFu, c, 0);
             const int s = c % kStages;
-            if (!mbar_wait(&sh.full[s], (c / kStages) & 1)) {
+            // A parity wait only tells the current phase from the one before it.  Copies complete out of
+            // order, so this warp can get here while the chunk that used the stage one lap earlier
+            // (c - kStages) is still in flight; the barrier is then a whole phase behind and the wait
+            // passes at once.  The stage's record number says which chunk the stage really holds: the
+            // wait is over only when it is this chunk's (the producer writes it before it arrives on the
+            // barrier, and cannot write it before the earlier chunk has been released).
+            bool landed = false;
+            for (uint32_t spin = 0; spin < kWaitLimit; ++spin) {
+                if (!mbar_wait(&sh.full[s], (c / kStages) & 1)) break;  // the bounded wait ran out
+                if (*reinterpret_cast<volatile int32_t*>(&sh.c_rec[s]) == static_cast<int32_t>(c)) {
+                    landed = true;
+                    break;
+                }
+            }
+            if (!landed) {
                 atomicExch(&status->timeout, 1);
                 sh.abort = 1;
-                mbar_wait(&sh.full[s], (c / kStages) & 1);  // nothing may still be landing when the CTA leaves
                 break;  // no barrier ties this warp to the others: it can simply leave
             }
             const int slot = sh.c_slot[s];
@@ -601,28 +572,25 @@ score_ring_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
             const int tail = static_cast<int>((head + row_bytes) & 15);  // bytes of the row in its last vector (0 = all 16)
             const int e0 = -head / static_cast<int>(sizeof(T));          // element index of slot 0 of vector 0
             const uint4* vec = reinterpret_cast<const uint4*>(bufs + static_cast<size_t>(s) * kChunkBytes);
+            // vector of the true-class logit within the row; it may be one of the two edge vectors
+            const int64_t ey = rs.label - e0;  // element slot counted from the row's first vector
+            const int vy = static_cast<int>(ey / EPV);
 
-            // -- the chunk into registers; the two ends of a row need care
+            // -- the chunk into registers: whole vectors of the row only, nothing to mask
             uint4 raw[kVecPerLane];
-            const uint32_t ninf = EPV == 4 ? 0xFF800000u : 0xFF80FF80u;
-            const int last_i = (tail && v0 + nv == nvec) ? nv - 1 : -1;  // where the row ends inside a vector
+            if (nv == kChunkVecs) {
 #pragma unroll
-            for (int u = 0; u < kVecPerLane; ++u) {
-                const int i = lane + 32 * u;
-                raw[u] = i < nv ? vec[i] : make_uint4(ninf, ninf, ninf, ninf);
-                if (i == last_i)
-                    raw[u] = row == rows - 1 ? ragged_vector<T>(logits, row, C, e0 + (nvec - 1) * EPV)
-                                             : mask_outside<T>(raw[u], 0, tail / static_cast<int>(sizeof(T)));
+                for (int u = 0; u < kVecPerLane; ++u) raw[u] = vec[lane + 32 * u];
+            } else {  // the last chunk of a row
+                const uint32_t ninf = EPV == 4 ? 0xFF800000u : 0xFF80FF80u;
+#pragma unroll
+                for (int u = 0; u < kVecPerLane; ++u) {
+                    const int i = lane + 32 * u;
+                    raw[u] = i < nv ? vec[i] : make_uint4(ninf, ninf, ninf, ninf);
+                }
             }
-            if (lane == 0 && v0 == 0 && head)  // the row starts inside its first vector
-                raw[0] = row == 0 ? ragged_vector<T>(logits, row, C, e0) : mask_outside<T>(raw[0], -e0, EPV);
-            {  // the true-class logit, if this chunk holds it
-                const int64_t ey = rs.label - e0;  // element slot within the row's vectors
-                const int vy = static_cast<int>(ey / EPV);
-                if (lane == 0 && vy >= v0 && vy < v0 + nv)
-                    rs.xy = (row == 0 || row == rows - 1) ? Elem<T>::widen(logits[row * C + rs.label])
-                                                          : Elem<T>::widen(reinterpret_cast<const T*>(vec)[ey - static_cast<int64_t>(v0) * EPV]);
-            }
+            if (lane == 0 && vy >= v0 && vy < v0 + nv)  // the true-class logit, if this chunk holds it
+                rs.xy = Elem<T>::widen(reinterpret_cast<const T*>(vec)[ey - static_cast<int64_t>(v0) * EPV]);
 
             // -- chunk maximum (every lane's loads have returned once the shuffles are through)
             VecMax<T> vm;
@@ -659,9 +627,26 @@ score_ring_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
             const float Mb = ib < nrec ? sh.rec_max[(first + ib) % kRecSlots] : neg_inf();
             const float Sa = ia < nrec ? sh.rec_sum[(first + ia) % kRecSlots] : 0.f;
             const float Sb = ib < nrec ? sh.rec_sum[(first + ib) % kRecSlots] : 0.f;
-            const float m = warp_max(fmaxf(Ma, Mb));
-            const float ssum = warp_sum(Sa * ex2((Ma - m) * kLog2e) + Sb * ex2((Mb - m) * kLog2e));
-            const float xy = rs.xy;
+            // the elements of the (at most two) vectors in which the row starts and ends: lanes 0..7 take the
+            // first vector's slots, lanes 8..15 the last vector's, one element load each
+            float xe = neg_inf();
+            int64_t je = -1;
+            if (lane < 16) {
+                const int slot_e = lane & 7;
+                const bool at_head = lane < 8;
+                if (slot_e < EPV && (at_head ? head != 0 : tail != 0)) {
+                    const int64_t j = e0 + (at_head ? 0 : static_cast<int64_t>(nvec - 1) * EPV) + slot_e;
+                    if (j >= 0 && j < C) {
+                        je = j;
+                        xe = Elem<T>::widen(logits[row * C + j]);
+                    }
+                }
+            }
+            const float m = warp_max(fmaxf(fmaxf(Ma, Mb), xe));
+            const float ssum = warp_sum(Sa * ex2((Ma - m) * kLog2e) + Sb * ex2((Mb - m) * kLog2e) +
+                                        (je >= 0 ? ex2((xe - m) * kLog2e) : 0.f));
+            const bool y_at_edge = (head && vy == 0) || (tail && vy == nvec - 1);
+            const float xy = y_at_edge ? warp_max(je == rs.label ? xe : neg_inf()) : rs.xy;
             float loss;
             if (ssum >= 1.5f) {
                 loss = (m - xy) + logf(ssum);
