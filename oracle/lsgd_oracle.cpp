@@ -12,8 +12,15 @@
 // Pins (checked by the CPU test-suite against facts that do not come from this
 // file): closed forms ln C / softplus / C = 1, shift and permutation invariance,
 // a library log-sum-exp, brute-force selection, one-hot / uniform / (32,1)-step
-// weights.  Ordering of NaN, +-0 and all-ignored samples is a convention of this
-// library, not of the paper: parity unpinned for those cases (convention only).
+// weights; for the per-epoch data allocation, the generator's published known
+// answers, the paper's own (32, 8, 1, 2) setting for the sizes, and the
+// statistics that "uniformly without replacement" fixes (valid subsets, every
+// subset equally likely, uniform and independent priorities).  Ordering of NaN,
+// +-0 and all-ignored samples is a convention of this library, not of the
+// paper: parity unpinned for those cases (convention only).  The same holds for
+// which random stream feeds a draw (counter layout, 30-bit priorities, ties by
+// lower index): the paper only says "randomly"; the distribution is pinned, the
+// particular bits are this library's convention.
 #include <algorithm>
 #include <cmath>
 #include <cstdint>
@@ -138,6 +145,126 @@ int oracle_weights_from_steps(const int32_t* tau, int32_t P, float* w_out) {
     if (!(total > 0.0)) return 1;
     for (int32_t i = 0; i < P; ++i) w_out[i] = static_cast<float>(static_cast<double>(tau[i]) / total);
     return 0;
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------------
+// Per-epoch data allocation (Section 4.2; Algorithm 1, the four steps before the
+// training loop).
+// ---------------------------------------------------------------------------
+namespace {
+
+// Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw: "Parallel random
+// numbers: as easy as 1, 2, 3", SC'11): a 128-bit counter and a 64-bit key give
+// four 32-bit words.  One round multiplies words 0 and 2 of the counter by two
+// fixed odd constants, swaps the product halves into place and mixes the key in;
+// the key is advanced by two Weyl constants between rounds.
+void philox4x32_10(const uint32_t ctr_in[4], const uint32_t key_in[2], uint32_t out[4]) {
+    const uint64_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+    const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    uint32_t c[4] = {ctr_in[0], ctr_in[1], ctr_in[2], ctr_in[3]};
+    uint32_t k0 = key_in[0], k1 = key_in[1];
+    for (int round = 0; round < 10; ++round) {
+        const uint64_t p0 = M0 * c[0], p1 = M1 * c[2];
+        const uint32_t hi0 = static_cast<uint32_t>(p0 >> 32), lo0 = static_cast<uint32_t>(p0);
+        const uint32_t hi1 = static_cast<uint32_t>(p1 >> 32), lo1 = static_cast<uint32_t>(p1);
+        const uint32_t n0 = hi1 ^ c[1] ^ k0, n1 = lo1, n2 = hi0 ^ c[3] ^ k1, n3 = lo0;
+        c[0] = n0; c[1] = n1; c[2] = n2; c[3] = n3;
+        k0 += W0;
+        k1 += W1;
+    }
+    for (int i = 0; i < 4; ++i) out[i] = c[i];
+}
+
+// Random priority of sample i in draw `stream` under `seed`: 30 bits.  Samples
+// 4j .. 4j+3 share one Philox block: counter (j, 0, stream_lo, stream_hi), key
+// (seed_lo, seed_hi); sample i takes word i mod 4, top 30 bits.
+uint32_t priority_of(int64_t i, uint64_t seed, uint64_t stream) {
+    const uint32_t ctr[4] = {static_cast<uint32_t>(i >> 2), 0u, static_cast<uint32_t>(stream),
+                             static_cast<uint32_t>(stream >> 32)};
+    const uint32_t key[2] = {static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32)};
+    uint32_t w[4];
+    philox4x32_10(ctr, key, w);
+    return w[i & 3] >> 2;
+}
+
+}  // namespace
+
+extern "C" {
+
+int oracle_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) {
+    philox4x32_10(ctr, key, out);
+    return 0;
+}
+
+// Section 4.2: of N samples per epoch the fast workers get
+//   N_F = tau_F P_F / (tau_F P_F + tau_S P_S) * N   (rounded down),
+// the slow workers the rest, N_S = N - N_F (so that one epoch covers N samples),
+// and k = lambda * N_F (rounded down, evaluated in double) of the fast workers'
+// samples are the highest-loss ones.
+int oracle_allocation_sizes(int64_t N, int32_t tau_f, int32_t p_f, int32_t tau_s, int32_t p_s, double lambda,
+                            int64_t* n_fast, int64_t* n_slow, int64_t* k_high) {
+    if (N < 0 || tau_f < 0 || p_f < 0 || tau_s < 0 || p_s < 0 || !(lambda >= 0.0 && lambda <= 1.0)) return 1;
+    const __int128 a = static_cast<__int128>(tau_f) * p_f, b = static_cast<__int128>(tau_s) * p_s;
+    if (a + b == 0) return 1;
+    const int64_t nf = static_cast<int64_t>(a * N / (a + b));
+    *n_fast = nf;
+    *n_slow = N - nf;
+    int64_t k = static_cast<int64_t>(std::floor(lambda * static_cast<double>(nf)));
+    *k_high = std::min(std::max<int64_t>(k, 0), nf);
+    return 0;
+}
+
+// "Evenly distribute" a list of n entries over P workers: worker p gets the
+// contiguous range [floor(p n / P), floor((p+1) n / P)), so shares differ by at
+// most one entry and together cover the list once.
+int oracle_worker_share(int64_t n, int32_t P, int32_t p, int64_t* begin, int64_t* end) {
+    if (n < 0 || P < 1 || p < 0 || p >= P) return 1;
+    *begin = static_cast<int64_t>(static_cast<__int128>(n) * p / P);
+    *end = static_cast<int64_t>(static_cast<__int128>(n) * (p + 1) / P);
+    return 0;
+}
+
+// Uniform sampling without replacement (Section 4.2: "randomly selected from the
+// rest of data", "randomly sampled from the total N samples without
+// replacement"): every sample gets an independent random priority; the draw is
+// the m candidates with the highest priority (ties: lower index), listed in that
+// order.  Candidates are the indices 0..N-1 that are not in exclude_idx.
+// Independent, identically distributed priorities make every m-subset of the
+// candidates equally likely and the listed order a uniform random order.
+int oracle_draw_uniform(int64_t N, int64_t m, uint64_t seed, uint64_t stream, const int32_t* exclude_idx,
+                        int64_t n_exclude, int32_t* out_idx) {
+    std::vector<char> excluded(static_cast<size_t>(N), 0);
+    for (int64_t j = 0; j < n_exclude; ++j)
+        if (exclude_idx[j] >= 0 && exclude_idx[j] < N) excluded[static_cast<size_t>(exclude_idx[j])] = 1;
+    std::vector<int32_t> cand;
+    for (int64_t i = 0; i < N; ++i)
+        if (!excluded[static_cast<size_t>(i)]) cand.push_back(static_cast<int32_t>(i));
+    if (m < 0 || m > static_cast<int64_t>(cand.size())) return 1;
+    std::vector<uint32_t> pri(static_cast<size_t>(N));
+    for (int64_t i = 0; i < N; ++i) pri[static_cast<size_t>(i)] = priority_of(i, seed, stream);
+    std::stable_sort(cand.begin(), cand.end(), [&](int32_t a, int32_t b) { return pri[a] > pri[b]; });
+    for (int64_t j = 0; j < m; ++j) out_idx[j] = cand[static_cast<size_t>(j)];
+    return 0;
+}
+
+// The priorities themselves (for the tests' statistics).
+int oracle_priorities(int64_t N, uint64_t seed, uint64_t stream, uint32_t* out) {
+    for (int64_t i = 0; i < N; ++i) out[i] = priority_of(i, seed, stream);
+    return 0;
+}
+
+// Data allocation for the fast workers (Section 4.2; Algorithm 1, "select ...
+// high-loss samples" then "fill the remainder ... by randomly sampling from the
+// unselected samples"): the k highest-loss samples in loss-descending order,
+// followed by n_fill samples drawn uniformly without replacement from the other
+// N - k.
+int oracle_fast_allocation(const float* losses, int64_t N, int64_t k, int64_t n_fill, uint64_t seed, uint64_t stream,
+                           int32_t* out_idx) {
+    if (k < 0 || n_fill < 0 || k + n_fill > N) return 1;
+    if (oracle_topk(losses, N, k, 0, out_idx, nullptr) != 0) return 1;
+    return oracle_draw_uniform(N, n_fill, seed, stream, out_idx, k, out_idx + k);
 }
 
 }  // extern "C"

@@ -40,7 +40,16 @@ def _load():
         lib.oracle_topk.argtypes = [vp, i64, i64, ctypes.c_int, vp, vp]
         lib.oracle_aggregate.argtypes = [vp, vp, i32, i64, vp, vp, vp]
         lib.oracle_weights_from_steps.argtypes = [vp, i32, vp]
-        for f in (lib.oracle_score, lib.oracle_topk, lib.oracle_aggregate, lib.oracle_weights_from_steps):
+        u64, dbl = ctypes.c_uint64, ctypes.c_double
+        lib.oracle_philox4x32_10.argtypes = [vp, vp, vp]
+        lib.oracle_allocation_sizes.argtypes = [i64, i32, i32, i32, i32, dbl, vp, vp, vp]
+        lib.oracle_worker_share.argtypes = [i64, i32, i32, vp, vp]
+        lib.oracle_draw_uniform.argtypes = [i64, i64, u64, u64, vp, i64, vp]
+        lib.oracle_priorities.argtypes = [i64, u64, u64, vp]
+        lib.oracle_fast_allocation.argtypes = [vp, i64, i64, i64, u64, u64, vp]
+        for f in (lib.oracle_score, lib.oracle_topk, lib.oracle_aggregate, lib.oracle_weights_from_steps,
+                  lib.oracle_philox4x32_10, lib.oracle_allocation_sizes, lib.oracle_worker_share,
+                  lib.oracle_draw_uniform, lib.oracle_priorities, lib.oracle_fast_allocation):
             f.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -110,3 +119,58 @@ def weights_from_steps(tau) -> np.ndarray:
     if rc != 0:
         raise ValueError("step counts must sum to a positive number")
     return w
+
+
+def philox4x32_10(ctr, key) -> np.ndarray:
+    """One Philox4x32-10 block: ctr (4 x u32), key (2 x u32) -> 4 x u32."""
+    c = np.ascontiguousarray(ctr, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    out = np.empty(4, dtype=np.uint32)
+    assert c.size == 4 and k.size == 2
+    _load().oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def allocation_sizes(N: int, tau_fast: int, p_fast: int, tau_slow: int, p_slow: int, lam: float):
+    """(N_F, N_S, k) of Section 4.2."""
+    out = np.zeros(3, dtype=np.int64)
+    rc = _load().oracle_allocation_sizes(N, tau_fast, p_fast, tau_slow, p_slow, lam, _ptr(out[0:1]), _ptr(out[1:2]),
+                                         _ptr(out[2:3]))
+    if rc != 0:
+        raise ValueError("invalid allocation arguments")
+    return int(out[0]), int(out[1]), int(out[2])
+
+
+def worker_share(n: int, P: int, p: int):
+    """[begin, end) of worker p's part of an n-entry list split evenly over P workers."""
+    out = np.zeros(2, dtype=np.int64)
+    rc = _load().oracle_worker_share(n, P, p, _ptr(out[0:1]), _ptr(out[1:2]))
+    if rc != 0:
+        raise ValueError("invalid split arguments")
+    return int(out[0]), int(out[1])
+
+
+def draw_uniform(N: int, m: int, seed: int, stream: int, exclude=None) -> np.ndarray:
+    """m indices drawn uniformly without replacement from 0..N-1 minus `exclude`, in draw order."""
+    ex = np.ascontiguousarray(exclude if exclude is not None else [], dtype=np.int32)
+    out = np.empty(m, dtype=np.int32)
+    rc = _load().oracle_draw_uniform(N, m, seed, stream, _ptr(ex), ex.size, _ptr(out))
+    if rc != 0:
+        raise ValueError("more draws than candidates")
+    return out
+
+
+def priorities(N: int, seed: int, stream: int) -> np.ndarray:
+    out = np.empty(N, dtype=np.uint32)
+    _load().oracle_priorities(N, seed, stream, _ptr(out))
+    return out
+
+
+def fast_allocation(losses: np.ndarray, k: int, n_fill: int, seed: int, stream: int) -> np.ndarray:
+    """The fast workers' samples: k highest-loss first, then n_fill drawn from the rest."""
+    losses = np.ascontiguousarray(losses, dtype=np.float32)
+    out = np.empty(k + n_fill, dtype=np.int32)
+    rc = _load().oracle_fast_allocation(_ptr(losses), losses.size, k, n_fill, seed, stream, _ptr(out))
+    if rc != 0:
+        raise ValueError("k + n_fill exceeds N")
+    return out
