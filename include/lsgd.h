@@ -165,6 +165,87 @@ LSGD_API lsgd_status lsgd_score_topk(const void* logits, lsgd_dtype dtype, const
                                      lsgd_order order, float* losses, int32_t* out_idx, float* out_vals,
                                      void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* ------------------------------------------------------------------------- */
+/* Per-epoch data allocation (Section 4.2, "Bias Injection via Data Sampling"; */
+/* Algorithm 1, the four steps before the training loop).                      */
+/* ------------------------------------------------------------------------- */
+
+/*
+ * lsgd_allocation_sizes — how many of the N samples of an epoch each worker
+ * group gets (Section 4.2): with P_F fast workers doing tau_F local steps per
+ * round and P_S slow workers doing tau_S,
+ *     N_F = floor(N * tau_F P_F / (tau_F P_F + tau_S P_S)),   N_S = N - N_F,
+ *     k   = floor(lambda * N_F)      (the high-loss part of the fast allocation),
+ * N_F in exact integer arithmetic, k in double.  The paper gives the ratios
+ * only; rounding N_F down and giving the slow workers the rest keeps one epoch
+ * at N samples.  Host only.  tau and P values >= 0 with tau_F P_F + tau_S P_S > 0
+ * and 0 <= lambda <= 1, else LSGD_ERR_INVALID_ARG.
+ *   n_fast, n_slow, k_high   host, out
+ */
+LSGD_API lsgd_status lsgd_allocation_sizes(int64_t N, int32_t tau_fast, int32_t p_fast, int32_t tau_slow,
+                                           int32_t p_slow, double lambda, int64_t* n_fast, int64_t* n_slow,
+                                           int64_t* k_high);
+
+/*
+ * lsgd_worker_share — "evenly distribute" a list of n sample indices over the
+ * P workers of a group (Section 4.2; Algorithm 1): worker p gets the contiguous
+ * entries [begin, end) = [floor(p n / P), floor((p + 1) n / P)).  Shares differ
+ * by at most one entry and cover the list exactly once.  Host only.
+ */
+LSGD_API lsgd_status lsgd_worker_share(int64_t n, int32_t P, int32_t p, int64_t* begin, int64_t* end);
+
+/*
+ * lsgd_draw_uniform — n_draw samples drawn uniformly at random, without
+ * replacement, from the samples 0..N-1 that are not listed in exclude_idx
+ * (Section 4.2: the slow workers' N_S samples "randomly sampled from the total
+ * N samples without replacement"; with an exclusion list, a draw "from the rest
+ * of data", e.g. the unified-sampling variant of the appendix where the slow
+ * workers draw from what the fast workers left).
+ *
+ * Every sample i gets the random priority q_i = top 30 bits of word (i mod 4)
+ * of the Philox4x32-10 block with counter (i div 4, 0, stream_lo, stream_hi) and
+ * key (seed_lo, seed_hi).  The draw is the n_draw candidates that come first in
+ * the order "higher q first, then lower index", written in that order: every
+ * subset is equally likely and the order is a uniform random order (up to ties
+ * among 30-bit priorities).  The same (N, seed, stream, exclusion) always gives
+ * the same result; different `stream` values give independent draws, so a
+ * caller can use e.g. stream = 2 * epoch for the fast group and 2 * epoch + 1
+ * for the slow group ("separated sampling").
+ *
+ *   exclude_idx  device, [n_exclude] int32 or NULL: distinct indices in [0, N)
+ *                (entries outside that range are ignored).
+ *   n_draw       0 <= n_draw <= N - n_exclude.
+ *   out_idx      device, [n_draw] int32.  May not overlap exclude_idx.
+ *   ws           device workspace of at least lsgd_draw_workspace_bytes(N, n_draw).
+ */
+LSGD_API size_t lsgd_draw_workspace_bytes(int64_t N, int64_t n_draw);
+LSGD_API lsgd_status lsgd_draw_uniform(int64_t N, int64_t n_draw, uint64_t seed, uint64_t stream,
+                                       const int32_t* exclude_idx, int64_t n_exclude, int32_t* out_idx, void* ws,
+                                       size_t ws_bytes, void* cuda_stream);
+
+/*
+ * lsgd_fast_allocation — the fast workers' samples for one epoch (Section 4.2,
+ * "Data Allocation for Fast Workers"; Algorithm 1: "select ... high-loss
+ * samples", then "fill the remainder ... by randomly sampling from the
+ * unselected samples"):
+ *     out_idx[0 .. k_high)               the k_high highest-loss samples, as
+ *                                        lsgd_topk_select gives them in
+ *                                        LSGD_ORDER_LOSS_DESC;
+ *     out_idx[k_high .. k_high + n_fill) n_fill samples drawn as by
+ *                                        lsgd_draw_uniform(seed, stream) with the
+ *                                        first part as the exclusion list.
+ * The list is then split over the fast workers with lsgd_worker_share.
+ *
+ *   losses   device, [N] fp32 (the loss table lsgd_score_losses writes).
+ *   k_high + n_fill <= N.      out_idx  device, [k_high + n_fill] int32.
+ *   ws       device workspace of at least
+ *            lsgd_fast_allocation_workspace_bytes(N, k_high, n_fill).
+ */
+LSGD_API size_t lsgd_fast_allocation_workspace_bytes(int64_t N, int64_t k_high, int64_t n_fill);
+LSGD_API lsgd_status lsgd_fast_allocation(const float* losses, int64_t N, int64_t k_high, int64_t n_fill,
+                                          uint64_t seed, uint64_t stream, int32_t* out_idx, void* ws,
+                                          size_t ws_bytes, void* cuda_stream);
+
 /*
  * lsgd_aggregate — biased model aggregation, Eq. 3:  out[j] = sum_i w_i * x_i[j]
  * over the P worker replicas' flattened parameters, accumulated in fp32 in

@@ -26,6 +26,8 @@ EXPORTS = (
     "lsgd_version", "lsgd_status_string", "lsgd_score_workspace_bytes", "lsgd_topk_workspace_bytes",
     "lsgd_score_topk_workspace_bytes", "lsgd_score_losses", "lsgd_topk_select", "lsgd_score_topk",
     "lsgd_aggregate", "lsgd_weights_from_steps", "lsgd_read_device_status", "lsgd_topk_select_static",
+    "lsgd_allocation_sizes", "lsgd_worker_share", "lsgd_draw_workspace_bytes", "lsgd_draw_uniform",
+    "lsgd_fast_allocation_workspace_bytes", "lsgd_fast_allocation",
 )
 STATIC_TOPK_MAX_N = 262144
 
@@ -60,10 +62,20 @@ def lib() -> ctypes.CDLL:
         L.lsgd_topk_select_static.restype = ci
         L.lsgd_score_topk.argtypes = [vp, ci, vp, i64, i64, i64, i64, i64, ci, vp, vp, vp, vp, sz, vp]
         L.lsgd_aggregate.argtypes = [vp, vp, i32, i64, vp, vp]
+        u64 = ctypes.c_uint64
+        L.lsgd_allocation_sizes.argtypes = [i64, i32, i32, i32, i32, ctypes.c_double, vp, vp, vp]
+        L.lsgd_worker_share.argtypes = [i64, i32, i32, vp, vp]
+        L.lsgd_draw_workspace_bytes.argtypes = [i64, i64]
+        L.lsgd_draw_workspace_bytes.restype = sz
+        L.lsgd_draw_uniform.argtypes = [i64, i64, u64, u64, vp, i64, vp, vp, sz, vp]
+        L.lsgd_fast_allocation_workspace_bytes.argtypes = [i64, i64, i64]
+        L.lsgd_fast_allocation_workspace_bytes.restype = sz
+        L.lsgd_fast_allocation.argtypes = [vp, i64, i64, i64, u64, u64, vp, vp, sz, vp]
         L.lsgd_weights_from_steps.argtypes = [vp, i32, vp]
         L.lsgd_read_device_status.argtypes = [vp, vp, vp]
         for name in ("lsgd_score_losses", "lsgd_topk_select", "lsgd_score_topk", "lsgd_aggregate",
-                     "lsgd_weights_from_steps", "lsgd_read_device_status"):
+                     "lsgd_weights_from_steps", "lsgd_read_device_status", "lsgd_allocation_sizes", "lsgd_worker_share",
+                     "lsgd_draw_uniform", "lsgd_fast_allocation"):
             getattr(L, name).restype = ci
         _lib = L
     return _lib
@@ -204,6 +216,59 @@ def aggregate(replicas, weights, out=None):
     st = lib().lsgd_aggregate(ctypes.cast(ptrs, ctypes.c_void_p), ctypes.cast(w, ctypes.c_void_p), P, D, _p(out), _stream())
     _check("lsgd_aggregate", st)
     return out
+
+
+def allocation_sizes(N: int, tau_fast: int, p_fast: int, tau_slow: int, p_slow: int, lam: float):
+    """lsgd_allocation_sizes: (N_F, N_S, k) of Section 4.2.  Host only."""
+    nf, ns, k = ctypes.c_int64(0), ctypes.c_int64(0), ctypes.c_int64(0)
+    st = lib().lsgd_allocation_sizes(N, tau_fast, p_fast, tau_slow, p_slow, lam, ctypes.byref(nf), ctypes.byref(ns),
+                                     ctypes.byref(k))
+    _check("lsgd_allocation_sizes", st)
+    return nf.value, ns.value, k.value
+
+
+def worker_share(n: int, P: int, p: int):
+    """lsgd_worker_share: [begin, end) of worker p's part of an n-entry list.  Host only."""
+    b, e = ctypes.c_int64(0), ctypes.c_int64(0)
+    _check("lsgd_worker_share", lib().lsgd_worker_share(n, P, p, ctypes.byref(b), ctypes.byref(e)))
+    return b.value, e.value
+
+
+def draw_workspace_bytes(N: int, n_draw: int) -> int:
+    return lib().lsgd_draw_workspace_bytes(N, n_draw)
+
+
+def fast_allocation_workspace_bytes(N: int, k_high: int, n_fill: int) -> int:
+    return lib().lsgd_fast_allocation_workspace_bytes(N, k_high, n_fill)
+
+
+def draw_uniform(N: int, n_draw: int, seed: int, stream: int, exclude_idx=None, out_idx=None, ws=None, device=None):
+    """lsgd_draw_uniform: n_draw of the N samples (minus exclude_idx), uniformly without replacement."""
+    dev = exclude_idx.device if exclude_idx is not None else (device or "cuda")
+    if out_idx is None:
+        out_idx = torch.empty(max(n_draw, 0), dtype=torch.int32, device=dev)
+    if ws is None:
+        ws = workspace(draw_workspace_bytes(N, n_draw), dev)
+    n_ex = exclude_idx.numel() if exclude_idx is not None else 0
+    if exclude_idx is not None and (exclude_idx.dtype != torch.int32 or not exclude_idx.is_contiguous()):
+        raise ValueError("exclude_idx must be a contiguous int32 tensor")
+    st = lib().lsgd_draw_uniform(N, n_draw, seed, stream, _p(exclude_idx), n_ex, _p(out_idx), _p(ws), ws.numel(), _stream())
+    _check("lsgd_draw_uniform", st)
+    return out_idx
+
+
+def fast_allocation(losses, k_high: int, n_fill: int, seed: int, stream: int, out_idx=None, ws=None):
+    """lsgd_fast_allocation: the k_high highest-loss samples, then n_fill drawn from the rest."""
+    N = losses.numel()
+    if losses.dtype != torch.float32 or not losses.is_contiguous():
+        raise ValueError("losses must be a contiguous float32 tensor")
+    if out_idx is None:
+        out_idx = torch.empty(max(k_high + n_fill, 0), dtype=torch.int32, device=losses.device)
+    if ws is None:
+        ws = workspace(fast_allocation_workspace_bytes(N, k_high, n_fill), losses.device)
+    st = lib().lsgd_fast_allocation(_p(losses), N, k_high, n_fill, seed, stream, _p(out_idx), _p(ws), ws.numel(), _stream())
+    _check("lsgd_fast_allocation", st)
+    return out_idx
 
 
 def weights_from_steps(tau) -> list[float]:

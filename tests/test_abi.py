@@ -27,7 +27,7 @@ def declared_symbols():
 
 def test_every_declared_symbol_is_exported(L):
     names = declared_symbols()
-    assert set(names) == set(L.EXPORTS) and len(names) == 12
+    assert set(names) == set(L.EXPORTS) and len(names) == 18
     lib = ctypes.CDLL(L.LIB_PATH)
     for n in names:
         assert getattr(lib, n) is not None
@@ -104,3 +104,44 @@ def test_argument_errors_are_found_before_any_cuda_call(L):
     assert lib.lsgd_score_losses(ptr, 0, ptr, 4, 1, 10, -100, big, ptr, 16, None) == L.ERR_WORKSPACE
     assert lib.lsgd_score_topk(ptr, 0, ptr, 4, 1, 10, -100, 5, 0, big, ptr, None, ptr, 1 << 20, None) == L.ERR_INVALID_ARG
     assert lib.lsgd_read_device_status(None, None, None) == L.ERR_INVALID_ARG
+
+
+def test_allocation_sizes_and_shares_host_only(L):
+    # Section 5.1's setting (tau_F = 32 on 8 fast workers, tau_S = 1 on 2 slow ones): N_F / N = 256 / 258
+    assert L.allocation_sizes(50_000, 32, 8, 1, 2, 1.0) == (49_612, 388, 49_612)
+    nf, ns, k = L.allocation_sizes(1_281_167, 16, 4, 4, 4, 0.3)
+    assert nf + ns == 1_281_167 and nf == 1_281_167 * 64 // 80 and k == int(0.3 * nf)
+    assert L.allocation_sizes(1000, 5, 0, 2, 3, 0.5) == (0, 1000, 0)
+    for bad in [(-1, 1, 1, 1, 1, 0.5), (10, 0, 0, 0, 0, 0.5), (10, 1, 1, 1, 1, 1.5), (10, 1, 1, 1, 1, float("nan")),
+                (10, -1, 1, 1, 1, 0.5)]:
+        with pytest.raises(L.LsgdError) as e:
+            L.allocation_sizes(*bad)
+        assert e.value.status == L.ERR_INVALID_ARG
+    parts = [L.worker_share(49_612, 8, p) for p in range(8)]
+    assert parts[0][0] == 0 and parts[-1][1] == 49_612 and all(parts[p][1] == parts[p + 1][0] for p in range(7))
+    assert {e - b for b, e in parts} <= {6201, 6202}
+    for bad in [(10, 0, 0), (10, 2, 2), (10, 2, -1), (-1, 2, 0)]:
+        with pytest.raises(L.LsgdError):
+            L.worker_share(*bad)
+
+
+def test_draw_argument_errors_are_found_before_any_cuda_call(L):
+    lib = L.lib()
+    ptr = ctypes.c_void_p(0x1000)
+    big = 1 << 24
+    assert L.draw_workspace_bytes(10, 11) == 0 and L.draw_workspace_bytes(-1, 0) == 0
+    assert L.draw_workspace_bytes(50_000, 388) >= L.topk_workspace_bytes(50_000, 388) + 4 * 50_000
+    assert L.fast_allocation_workspace_bytes(100, 60, 41) == 0
+    assert L.fast_allocation_workspace_bytes(50_000, 12_403, 37_209) == L.draw_workspace_bytes(50_000, 37_209)
+    assert lib.lsgd_draw_uniform(10, 11, 1, 0, None, 0, ptr, ptr, big, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_draw_uniform(10, 8, 1, 0, ptr, 3, ptr, ptr, big, None) == L.ERR_INVALID_ARG  # only 7 candidates
+    assert lib.lsgd_draw_uniform(10, 2, 1, 0, None, 3, ptr, ptr, big, None) == L.ERR_INVALID_ARG  # list missing
+    assert lib.lsgd_draw_uniform(10, 0, 1, 0, None, 0, None, None, 0, None) == L.OK
+    assert lib.lsgd_draw_uniform(1 << 31, 5, 1, 0, None, 0, ptr, ptr, big, None) == L.ERR_UNSUPPORTED
+    assert lib.lsgd_draw_uniform(10, 5, 1, 0, None, 0, ptr, ptr, 16, None) == L.ERR_WORKSPACE
+    assert lib.lsgd_draw_uniform(10, 5, 1, 0, None, 0, ctypes.c_void_p(0x1002), ptr, big, None) == L.ERR_ALIGNMENT
+    assert lib.lsgd_draw_uniform(10, 5, 1, 0, None, 0, ptr, ctypes.c_void_p(0x1010), big, None) == L.ERR_ALIGNMENT
+    assert lib.lsgd_fast_allocation(ptr, 10, 6, 5, 1, 0, ptr, ptr, big, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_fast_allocation(None, 10, 6, 2, 1, 0, ptr, ptr, big, None) == L.ERR_INVALID_ARG
+    assert lib.lsgd_fast_allocation(ptr, 10, 0, 0, 1, 0, None, None, 0, None) == L.OK
+    assert lib.lsgd_fast_allocation(ptr, 10, 6, 2, 1, 0, ptr, ptr, 16, None) == L.ERR_WORKSPACE
