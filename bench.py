@@ -332,33 +332,65 @@ def run_gpu(args, cfg):
     h_idx = torch.empty(cfg.k, dtype=torch.int32, pin_memory=True)
     h_vals = torch.empty(cfg.k, dtype=torch.float32, pin_memory=True)
     h_out = torch.empty(cfg.D, dtype=torch.float32, pin_memory=True)
-    h2d = h_logits.numel() * h_logits.element_size() + h_labels.numel() * 8 + cfg.P * cfg.D * 4
-    d2h = cfg.k * 8 + cfg.D * 4
+    h2d_st = h_logits.numel() * h_logits.element_size() + h_labels.numel() * 8
+    d2h_st = cfg.k * 8
+    h2d = h2d_st + cfg.P * cfg.D * 4
+    d2h = d2h_st + cfg.D * 4
 
-    def step_e2e():
+    def step_e2e(ev=None):
+        if ev:
+            ev[0].record()
         d_logits.copy_(h_logits, non_blocking=True)
         d_labels.copy_(h_labels, non_blocking=True)
-        for d, h in zip(d_reps, h_reps):
-            d.copy_(h, non_blocking=True)
         lsgd.score_topk(d_logits, d_labels, cfg.k, lsgd.ORDER_LOSS_DESC, losses=losses, out_idx=idx, out_vals=vals, ws=ws)
-        lsgd.aggregate(d_reps, weights, out=out)
         h_idx.copy_(idx, non_blocking=True)
         h_vals.copy_(vals, non_blocking=True)
+        if ev:
+            ev[1].record()
+        for d, h in zip(d_reps, h_reps):
+            d.copy_(h, non_blocking=True)
+        lsgd.aggregate(d_reps, weights, out=out)
         h_out.copy_(out, non_blocking=True)
+        if ev:
+            ev[2].record()
 
-    e2e_ms = float("nan")
+    e2e_ms = e2e_st_ms = float("nan")
     if not args.no_e2e:
         step_e2e()
         barrier()
-        s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        s2.record()
-        for _ in range(e2e_steps):
-            step_e2e()
-        e2.record()
+        e_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(e2e_steps)]
+        for i in range(e2e_steps):
+            step_e2e(e_ev[i])
         barrier()
-        e2e_ms = s2.elapsed_time(e2)
+        e2e_st_ms = float(sum(e[0].elapsed_time(e[1]) for e in e_ev))
+        e2e_ms = float(e_ev[0][0].elapsed_time(e_ev[-1][2]))
 
-    total_ms, st_sum, ag_sum, e2e_ms = max_over_ranks([total_ms, float(st_ms.sum()), float(ag_ms.sum()), e2e_ms], dev)
+    # ---- the epoch's data allocation (Section 4.2) on the loss table just written: fast workers' list
+    # (top-k + random fill) and the slow workers' independent draw, in the paper's 8-fast / 2-slow setting
+    n_fast, n_slow, _ = lsgd.allocation_sizes(cfg.N, 32, 8, 1, 2, 1.0)
+    k_high = min(cfg.k, n_fast)
+    n_fill = n_fast - k_high
+    a_idx = torch.empty(n_fast + n_slow, dtype=torch.int32, device=dev)
+    a_ws = lsgd.workspace(max(lsgd.fast_allocation_workspace_bytes(cfg.N, k_high, n_fill),
+                              lsgd.draw_workspace_bytes(cfg.N, n_slow)), dev)
+    a_steps = 20
+    a_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(a_steps)]
+    for i in range(3 + a_steps):
+        ev = a_ev[i - 3] if i >= 3 else None
+        if ev:
+            ev[0].record()
+        lsgd.fast_allocation(losses, k_high, n_fill, cfg.seed, 2 * i, out_idx=a_idx[:n_fast], ws=a_ws)
+        if ev:
+            ev[1].record()
+        lsgd.draw_uniform(cfg.N, n_slow, cfg.seed, 2 * i + 1, out_idx=a_idx[n_fast:], ws=a_ws)
+        if ev:
+            ev[2].record()
+    torch.cuda.synchronize()
+    fast_ms = float(np.median([e[0].elapsed_time(e[1]) for e in a_ev]))
+    slow_ms = float(np.median([e[1].elapsed_time(e[2]) for e in a_ev]))
+
+    total_ms, st_sum, ag_sum, e2e_ms, e2e_st_ms = max_over_ranks(
+        [total_ms, float(st_ms.sum()), float(ag_ms.sum()), e2e_ms, e2e_st_ms], dev)
     if rank == 0:
         peak, peak_src = measured_peak()
         st_bytes = score_topk_bytes(cfg, h_labels.numpy())
@@ -386,9 +418,17 @@ def run_gpu(args, cfg):
                                    "unit": "GB/s", "frac": ag_gbs / peak,
                                    "traffic": NCU_TRAFFIC_BYTES.get(("aggregate", cfg.cfg_id)) if not (args.n_samples or args.d_params) else None,
                                    "peak_source": peak_src},
-            "e2e": {"value": world * cfg.N * e2e_steps / (e2e_ms * 1e-3), "unit": "samples/s", "ms_per_step": e2e_ms / e2e_steps,
-                    "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "note": "whole step (score+top-k and aggregation) incl. copies; bound by the host link"},
+            "e2e": {"value": world * cfg.N * e2e_steps / (e2e_st_ms * 1e-3), "unit": "samples/s",
+                    "ms_per_step": e2e_st_ms / e2e_steps, "steps": e2e_steps,
+                    "h2d_bytes_per_step": h2d_st, "d2h_bytes_per_step": d2h_st,
+                    "note": "score+top-k with logits and labels copied from pinned host memory and the k indices and "
+                            "losses copied back, every step; bound by the host link",
+                    "whole_step": {"ms_per_step": e2e_ms / e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                                   "note": "adds the replicas' upload, the aggregation and the download of its result"}},
+            "allocation": {"n_fast": n_fast, "k_high": k_high, "n_fill": n_fill, "n_slow": n_slow,
+                           "fast_allocation_ms": fast_ms, "slow_draw_ms": slow_ms,
+                           "note": "Section 4.2 lists for 8 fast (tau 32) + 2 slow (tau 1) workers from the resident loss "
+                                   "table; median of 20 calls, outside the timed step"},
             "gpu_launches": n_launch * args.steps,
             "clocks": clocks.summary(),
             "input_generation_s": gen_s,

@@ -15,7 +15,9 @@
 // weights; for the per-epoch data allocation, the generator's published known
 // answers, the paper's own (32, 8, 1, 2) setting for the sizes, and the
 // statistics that "uniformly without replacement" fixes (valid subsets, every
-// subset equally likely, uniform and independent priorities).  Ordering of NaN,
+// subset equally likely, uniform and independent priorities); for the round
+// aggregation, the pinned Eq. 3 routine, float64 numpy, its fixed points and a
+// library's bf16 rounding.  Ordering of NaN,
 // +-0 and all-ignored samples is a convention of this library, not of the
 // paper: parity unpinned for those cases (convention only).  The same holds for
 // which random stream feeds a draw (counter layout, 30-bit priorities, ties by
@@ -265,6 +267,60 @@ int oracle_fast_allocation(const float* losses, int64_t N, int64_t k, int64_t n_
     if (k < 0 || n_fill < 0 || k + n_fill > N) return 1;
     if (oracle_topk(losses, N, k, 0, out_idx, nullptr) != 0) return 1;
     return oracle_draw_uniform(N, n_fill, seed, stream, out_idx, k, out_idx + k);
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------------
+// One round's aggregation as the training loop uses it (Section 2, the local-SGD
+// update rule; Eq. 3; Algorithm 1: every worker continues from x_{t+1}).
+// ---------------------------------------------------------------------------
+namespace {
+
+inline double replica_at(const void* rep, int dtype, int64_t j) {
+    if (dtype == 0) return static_cast<double>(static_cast<const float*>(rep)[j]);
+    return bf16_to_double(static_cast<const uint16_t*>(rep)[j]);
+}
+
+// fp32 -> bf16, round to nearest, ties to even (bf16 = the upper 16 bits of an fp32).
+inline uint16_t f32_to_bf16_rne(float f) {
+    uint32_t u;
+    std::memcpy(&u, &f, sizeof u);
+    if ((u & 0x7F800000u) == 0x7F800000u && (u & 0x007FFFFFu)) return static_cast<uint16_t>((u >> 16) | 0x0040u);  // NaN stays NaN
+    const uint32_t lower = u & 0xFFFFu, keep = u >> 16;
+    uint32_t r = keep;
+    if (lower > 0x8000u || (lower == 0x8000u && (keep & 1u))) r = keep + 1u;
+    return static_cast<uint16_t>(r);
+}
+
+}  // namespace
+
+extern "C" {
+
+// x_{t+1}[j] from the P replicas (fp32, or bf16 widened exactly), in double, ascending i:
+//   base == NULL:  sum_i w_i x_i[j]                          (Eq. 3)
+//   base != NULL:  base[j] + sum_i w_i (x_i[j] - base[j])    (the same update written around x_t = base, as in
+//                  Section 2's rule x_{t+1} = x_t - eta * (averaged local progress); equal to Eq. 3 when sum w = 1)
+// out (double), out_f32 (its rounding), out_bf16 (out_f32 rounded once more to bf16: what a bf16 replica holds after
+// the broadcast), abs_out (the error scale: sum_i |w_i x_i|, or sum_i |w_i (x_i - base)| in the delta form).  Any of
+// the four may be NULL.
+int oracle_aggregate_round(const void* const* replicas, int dtype, const float* w, int32_t P, int64_t D,
+                           const float* base, double* out, float* out_f32, uint16_t* out_bf16, double* abs_out) {
+    for (int64_t j = 0; j < D; ++j) {
+        const double b = base ? static_cast<double>(base[j]) : 0.0;
+        double acc = 0.0, mag = 0.0;
+        for (int32_t i = 0; i < P; ++i) {
+            const double term = static_cast<double>(w[i]) * (replica_at(replicas[i], dtype, j) - b);
+            acc += term;
+            mag += std::fabs(term);
+        }
+        const double r = b + acc;
+        if (out) out[j] = r;
+        if (out_f32) out_f32[j] = static_cast<float>(r);
+        if (out_bf16) out_bf16[j] = f32_to_bf16_rne(static_cast<float>(r));
+        if (abs_out) abs_out[j] = mag;
+    }
+    return 0;
 }
 
 }  // extern "C"

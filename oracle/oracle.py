@@ -47,6 +47,8 @@ def _load():
         lib.oracle_draw_uniform.argtypes = [i64, i64, u64, u64, vp, i64, vp]
         lib.oracle_priorities.argtypes = [i64, u64, u64, vp]
         lib.oracle_fast_allocation.argtypes = [vp, i64, i64, i64, u64, u64, vp]
+        lib.oracle_aggregate_round.argtypes = [vp, ctypes.c_int, vp, i32, i64, vp, vp, vp, vp, vp]
+        lib.oracle_aggregate_round.restype = ctypes.c_int
         for f in (lib.oracle_score, lib.oracle_topk, lib.oracle_aggregate, lib.oracle_weights_from_steps,
                   lib.oracle_philox4x32_10, lib.oracle_allocation_sizes, lib.oracle_worker_share,
                   lib.oracle_draw_uniform, lib.oracle_priorities, lib.oracle_fast_allocation):
@@ -174,3 +176,29 @@ def fast_allocation(losses: np.ndarray, k: int, n_fill: int, seed: int, stream: 
     if rc != 0:
         raise ValueError("k + n_fill exceeds N")
     return out
+
+
+def aggregate_round(replicas, weights: np.ndarray, base: np.ndarray | None = None):
+    """One round's aggregation in double: Eq. 3, or base + sum_i w_i (x_i - base) when `base` is given.
+
+    replicas: float32 arrays, or uint16 arrays holding bf16 bit patterns.  Returns (out float64, out rounded to
+    float32, that rounded to bf16 bits, error scale float64).
+    """
+    dt = F32 if replicas[0].dtype == np.float32 else BF16
+    want = np.float32 if dt == F32 else np.uint16
+    reps = [np.ascontiguousarray(r, dtype=want) for r in replicas]
+    P, D = len(reps), reps[0].size
+    assert all(r.size == D and r.dtype == want for r in reps)
+    w = np.ascontiguousarray(weights, dtype=np.float32)
+    assert w.size == P
+    b = np.ascontiguousarray(base, dtype=np.float32) if base is not None else None
+    assert b is None or b.size == D
+    ptrs = (ctypes.c_void_p * P)(*[r.ctypes.data for r in reps])
+    out = np.empty(D, dtype=np.float64)
+    out32 = np.empty(D, dtype=np.float32)
+    out16 = np.empty(D, dtype=np.uint16)
+    mag = np.empty(D, dtype=np.float64)
+    rc = _load().oracle_aggregate_round(ctypes.cast(ptrs, ctypes.c_void_p), dt, _ptr(w), P, D, _ptr(b), _ptr(out),
+                                        _ptr(out32), _ptr(out16), _ptr(mag))
+    assert rc == 0
+    return out, out32, out16, mag
