@@ -389,6 +389,29 @@ def run_gpu(args, cfg):
     fast_ms = float(np.median([e[0].elapsed_time(e[1]) for e in a_ev]))
     slow_ms = float(np.median([e[1].elapsed_time(e[2]) for e in a_ev]))
 
+    # ---- the round's aggregation as the training loop uses it: around x_t, written back into the replicas,
+    # fp32 and bf16 replicas (lsgd_aggregate_round); median of 10 calls each, outside the timed step
+    round_legs = {}
+    if not args.no_round:
+        d_base = torch.empty(cfg.D, dtype=torch.float32, device=dev)
+        d_base.copy_(d_reps[0])
+        d_reps16 = [r.to(torch.bfloat16) for r in d_reps]
+        for name, reps_, es, use_base, bcast in (("f32_delta_broadcast", d_reps, 4, True, True),
+                                                 ("bf16_plain", d_reps16, 2, False, False),
+                                                 ("bf16_delta_broadcast", d_reps16, 2, True, True)):
+            r_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(10)]
+            for i in range(13):
+                if i >= 3:
+                    r_ev[i - 3][0].record()
+                lsgd.aggregate_round(reps_, weights, base=d_base if use_base else None, out=out, broadcast=bcast)
+                if i >= 3:
+                    r_ev[i - 3][1].record()
+            torch.cuda.synchronize()
+            ms = float(np.median([e[0].elapsed_time(e[1]) for e in r_ev]))
+            nbytes = cfg.D * (cfg.P * es * (2 if bcast else 1) + (4 if use_base else 0) + 4)
+            round_legs[name] = {"ms": ms, "algorithmic_bytes": nbytes, "gbs": nbytes / ms / 1e6}
+        del d_reps16, d_base
+
     total_ms, st_sum, ag_sum, e2e_ms, e2e_st_ms = max_over_ranks(
         [total_ms, float(st_ms.sum()), float(ag_ms.sum()), e2e_ms, e2e_st_ms], dev)
     if rank == 0:
@@ -429,6 +452,7 @@ def run_gpu(args, cfg):
                            "fast_allocation_ms": fast_ms, "slow_draw_ms": slow_ms,
                            "note": "Section 4.2 lists for 8 fast (tau 32) + 2 slow (tau 1) workers from the resident loss "
                                    "table; median of 20 calls, outside the timed step"},
+            "aggregation_round": round_legs,
             "gpu_launches": n_launch * args.steps,
             "clocks": clocks.summary(),
             "input_generation_s": gen_s,
@@ -459,6 +483,7 @@ def main():
     ap.add_argument("--config", type=int, default=4, choices=sorted(wl.CONFIGS))
     ap.add_argument("--impl", default="lsgd", choices=["lsgd", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-round", action="store_true", help="skip the lsgd_aggregate_round legs (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--n-samples", type=int, default=0, help="profiling: shrink the pool to this many samples")
     ap.add_argument("--d-params", type=int, default=0, help="profiling: shrink each replica to this many parameters")

@@ -267,6 +267,33 @@ LSGD_API lsgd_status lsgd_aggregate(const float* const* replicas, const float* w
                                     int64_t D, float* out, void* cuda_stream);
 
 /*
+ * lsgd_aggregate_round — the aggregation step as one round of the training loop
+ * needs it (Eq. 3; the local-SGD update rule of Section 2; Algorithm 1: after
+ * "Aggregate the local models" every worker continues from x_{t+1}):
+ *
+ *   base == NULL:  x_{t+1}[j] = sum_i w_i x_i[j]                         (Eq. 3)
+ *   base != NULL:  x_{t+1}[j] = base[j] + sum_i w_i (x_i[j] - base[j])   (Eq. 3 written around base = x_t, the
+ *                  form of Section 2's rule "x_t minus the averaged local progress"; identical to Eq. 3 when the
+ *                  weights sum to one, and more accurate in fp32 because the differences are small)
+ *
+ * accumulated in fp32 in ascending i (differences first, one multiply, fused multiply-adds, the base added last).
+ * The result is written to `out` (fp32) and, if `broadcast` is non-zero, also into every replica, rounded to the
+ * replicas' type (bf16: round to nearest even), all in the one pass that reads them.
+ *
+ *   replicas   HOST array of P DEVICE pointers, each to D values of type `dtype` (LSGD_F32 or LSGD_BF16), aligned
+ *              to the element size (16-byte alignment of every pointer takes the vectorised path).  Read before the
+ *              call returns.  Overwritten on the device when broadcast != 0.
+ *   weights    HOST, P fp32, used as given (not normalised).      1 <= P <= LSGD_MAX_REPLICAS,  D >= 0.
+ *   base       device, [D] fp32, or NULL.
+ *   out        device, [D] fp32, or NULL when broadcast != 0 (the replicas then hold the result).
+ *   Aliasing: `out` may be exactly `base`, and for fp32 replicas `out` or `base` may be exactly one replica; any
+ *   partial overlap, and with broadcast any overlap between two replicas, is LSGD_ERR_INVALID_ARG.
+ */
+LSGD_API lsgd_status lsgd_aggregate_round(void* const* replicas, lsgd_dtype dtype, const float* weights, int32_t P,
+                                          int64_t D, const float* base, float* out, int32_t broadcast,
+                                          void* cuda_stream);
+
+/*
  * lsgd_weights_from_steps — the weights of Eq. 3, w_i = tau_i / sum_j tau_j, from
  * the local step counts tau_i of the P workers.  Host only; computed in double
  * and rounded once to fp32.  tau_i >= 0 and sum > 0, else LSGD_ERR_INVALID_ARG.

@@ -27,7 +27,7 @@ EXPORTS = (
     "lsgd_score_topk_workspace_bytes", "lsgd_score_losses", "lsgd_topk_select", "lsgd_score_topk",
     "lsgd_aggregate", "lsgd_weights_from_steps", "lsgd_read_device_status", "lsgd_topk_select_static",
     "lsgd_allocation_sizes", "lsgd_worker_share", "lsgd_draw_workspace_bytes", "lsgd_draw_uniform",
-    "lsgd_fast_allocation_workspace_bytes", "lsgd_fast_allocation",
+    "lsgd_fast_allocation_workspace_bytes", "lsgd_fast_allocation", "lsgd_aggregate_round",
 )
 STATIC_TOPK_MAX_N = 262144
 
@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.lsgd_topk_select_static.restype = ci
         L.lsgd_score_topk.argtypes = [vp, ci, vp, i64, i64, i64, i64, i64, ci, vp, vp, vp, vp, sz, vp]
         L.lsgd_aggregate.argtypes = [vp, vp, i32, i64, vp, vp]
+        L.lsgd_aggregate_round.argtypes = [vp, ci, vp, i32, i64, vp, vp, i32, vp]
+        L.lsgd_aggregate_round.restype = ci
         u64 = ctypes.c_uint64
         L.lsgd_allocation_sizes.argtypes = [i64, i32, i32, i32, i32, ctypes.c_double, vp, vp, vp]
         L.lsgd_worker_share.argtypes = [i64, i32, i32, vp, vp]
@@ -215,6 +217,28 @@ def aggregate(replicas, weights, out=None):
         raise ValueError("one weight per replica")
     st = lib().lsgd_aggregate(ctypes.cast(ptrs, ctypes.c_void_p), ctypes.cast(w, ctypes.c_void_p), P, D, _p(out), _stream())
     _check("lsgd_aggregate", st)
+    return out
+
+
+def aggregate_round(replicas, weights, base=None, out=None, broadcast: bool = False, want_out: bool = True):
+    """lsgd_aggregate_round: Eq. 3 (around `base` if given) over fp32 or bf16 replicas; optionally written back into them."""
+    P = len(replicas)
+    D = replicas[0].numel() if P else 0
+    dt = _dtype_code(replicas[0]) if P else F32
+    for r in replicas:
+        if r.dtype != replicas[0].dtype or r.numel() != D or not r.is_contiguous():
+            raise ValueError("replicas must be contiguous tensors of one dtype and size")
+    if len(weights) != P:
+        raise ValueError("one weight per replica")
+    if base is not None and (base.dtype != torch.float32 or base.numel() != D or not base.is_contiguous()):
+        raise ValueError("base must be a contiguous float32 tensor of D elements")
+    if out is None and (want_out or not broadcast):
+        out = torch.empty(D, dtype=torch.float32, device=replicas[0].device)
+    ptrs = (ctypes.c_void_p * max(P, 1))(*[r.data_ptr() for r in replicas])
+    w = (ctypes.c_float * max(P, 1))(*[float(x) for x in weights])
+    st = lib().lsgd_aggregate_round(ctypes.cast(ptrs, ctypes.c_void_p), dt, ctypes.cast(w, ctypes.c_void_p), P, D, _p(base),
+                                    _p(out), 1 if broadcast else 0, _stream())
+    _check("lsgd_aggregate_round", st)
     return out
 
 

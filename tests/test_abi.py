@@ -27,7 +27,7 @@ def declared_symbols():
 
 def test_every_declared_symbol_is_exported(L):
     names = declared_symbols()
-    assert set(names) == set(L.EXPORTS) and len(names) == 18
+    assert set(names) == set(L.EXPORTS) and len(names) == 19
     lib = ctypes.CDLL(L.LIB_PATH)
     for n in names:
         assert getattr(lib, n) is not None
@@ -145,3 +145,28 @@ def test_draw_argument_errors_are_found_before_any_cuda_call(L):
     assert lib.lsgd_fast_allocation(None, 10, 6, 2, 1, 0, ptr, ptr, big, None) == L.ERR_INVALID_ARG
     assert lib.lsgd_fast_allocation(ptr, 10, 0, 0, 1, 0, None, None, 0, None) == L.OK
     assert lib.lsgd_fast_allocation(ptr, 10, 6, 2, 1, 0, ptr, ptr, 16, None) == L.ERR_WORKSPACE
+
+
+def test_aggregate_round_argument_errors(L):
+    lib = L.lib()
+    one = ctypes.c_float(1.0)
+    wp = ctypes.cast(ctypes.pointer(one), ctypes.c_void_p)
+    two = (ctypes.c_float * 2)(0.5, 0.5)
+    w2 = ctypes.cast(two, ctypes.c_void_p)
+    arr = (ctypes.c_void_p * 1)(0x10000)
+    arrp = ctypes.cast(arr, ctypes.c_void_p)
+    far = ctypes.c_void_p(0x90000)
+    f = lib.lsgd_aggregate_round
+    assert f(arrp, 7, wp, 1, 16, None, far, 0, None) == L.ERR_UNSUPPORTED
+    assert f(arrp, 0, wp, 0, 16, None, far, 0, None) == L.ERR_INVALID_ARG
+    assert f(arrp, 0, wp, 1, 16, None, None, 0, None) == L.ERR_INVALID_ARG       # no destination at all
+    assert f(arrp, 0, wp, 1, 0, None, None, 1, None) == L.OK
+    assert f(arrp, 1, wp, 1, 16, None, ctypes.c_void_p(0x10000), 0, None) == L.ERR_INVALID_ARG  # bf16 replica aliasing fp32 out
+    assert f(arrp, 0, wp, 1, 16, None, ctypes.c_void_p(0x10010), 0, None) == L.ERR_INVALID_ARG  # partial overlap
+    assert f(arrp, 0, wp, 1, 16, ctypes.c_void_p(0x10020), far, 0, None) == L.ERR_INVALID_ARG   # base overlaps the replica
+    assert f(arrp, 0, wp, 1, 16, ctypes.c_void_p(0x90010), far, 0, None) == L.ERR_INVALID_ARG   # base overlaps out
+    assert f(arrp, 0, wp, 1, 16, None, ctypes.c_void_p(0x90002), 0, None) == L.ERR_ALIGNMENT
+    odd = (ctypes.c_void_p * 1)(0x10001)
+    assert f(ctypes.cast(odd, ctypes.c_void_p), 1, wp, 1, 16, None, far, 0, None) == L.ERR_ALIGNMENT
+    twice = (ctypes.c_void_p * 2)(0x10000, 0x10000)
+    assert f(ctypes.cast(twice, ctypes.c_void_p), 0, w2, 2, 16, None, far, 1, None) == L.ERR_INVALID_ARG  # broadcast into aliased replicas
