@@ -17,7 +17,12 @@ struct StatusBlock {
     int32_t bad_labels;   // tokens with a label outside [0, C) that is not ignore_index
     int32_t timeout;      // set when a bounded device-side wait ran out
     uint32_t row_ticket;  // dynamic row scheduler of the large-row scorer
-    uint32_t pad[61];
+    // Radix select: CTAs that finished histogram pass p take a ticket; the last one resolves digit p of the
+    // threshold key once for everybody: the key prefix with digits 0..p placed, and the rank left inside it.
+    uint32_t sel_done[3];
+    uint32_t sel_prefix[3];
+    uint32_t sel_want[3];
+    uint32_t pad[52];
 };
 static_assert(sizeof(StatusBlock) == 256, "status block is 256 bytes");
 
@@ -68,10 +73,34 @@ cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order or
 
 int sm_count();  // multiprocessors of the current device (cached per device)
 
+// Launches `kernel` so that it may be scheduled while the previous kernel of the stream is still draining
+// (programmatic dependent launch).  Such a kernel must call grid_dependency_wait() before it touches global
+// memory: that is where it waits for the previous kernel to have completed, with its writes visible.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(static_cast<unsigned>(block));
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---------------------------------------------------------------------------
 // Device helpers
 // ---------------------------------------------------------------------------
 #ifdef __CUDACC__
+
+// Programmatic dependent launch, device side.  grid_launch_dependents: the next kernel of the stream may start
+// being scheduled once every CTA of this grid has got here (or exited).  grid_dependency_wait: blocks until the
+// previous kernel has completed and its memory is visible; a no-op for a normally launched kernel.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // Order-preserving key of a loss: larger key = selected earlier.  -0 maps to +0,
 // every NaN maps to the largest key (it ranks above +inf).

@@ -16,6 +16,12 @@
 //      into the required tie-break.  Each scatter pass accumulates the digit
 //      counts of the next pass, so the sort is one kernel per digit.
 // Pools of at most kSmallN entries are sorted whole by a single CTA instead.
+//
+// The kernels are short and depend on one another, so their latency is what
+// counts: each digit of the threshold is resolved once, by the last CTA to
+// finish its histogram pass (a ticket, no waiting), and every kernel is launched
+// so that it can be scheduled while its predecessor drains (it waits for the
+// predecessor's completion before its first global access).
 #include <algorithm>
 
 #include "lsgd_internal.cuh"
@@ -111,18 +117,21 @@ __device__ void find_bin(const uint32_t* hist, int nbins, uint32_t& want, uint32
     // thread t owns bins [nbins - 1 - t*per - (per - 1), nbins - 1 - t*per], highest first
     uint32_t c[8];
     uint32_t sum = 0;
-    for (int i = 0; i < per; ++i) {
-        c[i] = hist[nbins - 1 - (threadIdx.x * per + i)];
-        sum += c[i];
-    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i)  // all loads in flight together
+        c[i] = i < per ? __ldcg(hist + (nbins - 1 - (threadIdx.x * per + i))) : 0u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) sum += c[i];
     const uint32_t before = block_exclusive_scan(sum, scratch);
     if (before < want && want <= before + sum) {
         uint32_t run = before;
-        for (int i = 0; i < per; ++i) {
-            if (want <= run + c[i]) {
+        bool found = false;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (!found && i < per && want <= run + c[i]) {
                 result[0] = nbins - 1 - (threadIdx.x * per + i);
                 result[1] = want - run;
-                break;
+                found = true;
             }
             run += c[i];
         }
@@ -131,6 +140,26 @@ __device__ void find_bin(const uint32_t* hist, int nbins, uint32_t& want, uint32
     bin = result[0];
     want = result[1];
     __syncthreads();
+}
+
+// After a histogram pass: the last CTA to get here resolves digit `pass` of the threshold from the finished
+// histogram and publishes (prefix, rank left) in the status block.  Every thread of the CTA must call it, after
+// its last atomic on the histogram.  `prefix_in`, `want_in`: the state before this digit.
+__device__ void publish_digit(StatusBlock* status, const uint32_t* hist, int pass, uint32_t prefix_in, uint32_t want_in,
+                              uint32_t* scratch, uint32_t* result) {
+    __shared__ uint32_t last_s;
+    __threadfence();  // this thread's histogram atomics are ordered before the ticket
+    __syncthreads();
+    if (threadIdx.x == 0) last_s = atomicAdd(&status->sel_done[pass], 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!last_s) return;
+    __threadfence();
+    uint32_t want = want_in, bin;
+    find_bin(hist + pass * kSelBins, pass == 2 ? 1024 : kSelBins, want, bin, scratch, result);
+    if (threadIdx.x == 0) {
+        status->sel_prefix[pass] = prefix_in | (pass == 0 ? bin << 21 : pass == 1 ? bin << 10 : bin);
+        status->sel_want[pass] = want;
+    }
 }
 
 // Resolves the digits of the threshold key that passes [0, upto) fixed.
@@ -173,16 +202,26 @@ __device__ __forceinline__ void load_keys(const float* __restrict__ losses, int6
     }
 }
 
-// Histogram pass `pass`: counts digit `pass` of the keys that match the prefix
-// fixed by the earlier passes.
+// Histogram pass `pass`: counts digit `pass` of the keys that match the prefix fixed by the earlier passes, then
+// (last CTA) resolves that digit.  `prev_published`: the state after the previous pass is in the status block;
+// otherwise (pass 1 after a scorer that built the first histogram itself) digit 0 is resolved here by every CTA.
 __global__ void __launch_bounds__(kThreads)
-select_hist_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, int pass, uint32_t* hist) {
+select_hist_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, int pass, bool prev_published,
+                   uint32_t* hist, StatusBlock* status) {
     __shared__ uint32_t hist_s[kSelBins];
     __shared__ uint32_t scratch[kThreads / 32 + 1];
     __shared__ uint32_t result[2];
     for (int i = threadIdx.x; i < kSelBins; i += kThreads) hist_s[i] = 0;
-    uint32_t want;
-    const uint32_t prefix = resolve_prefix(hist, pass, k, want, scratch, result);
+    grid_dependency_wait();
+    uint32_t want = k, prefix = 0;
+    if (pass > 0) {
+        if (prev_published) {
+            prefix = __ldcg(&status->sel_prefix[pass - 1]);
+            want = __ldcg(&status->sel_want[pass - 1]);
+        } else {
+            prefix = resolve_prefix(hist, pass, k, want, scratch, result);
+        }
+    }
     __syncthreads();
     const uint32_t mask = prefix_mask(pass);
     for (int64_t tile = blockIdx.x; tile * kTile < N; tile += gridDim.x) {
@@ -209,20 +248,19 @@ select_hist_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, int 
         }
     }
     __syncthreads();
+    grid_launch_dependents();  // only the flush and the digit's resolution are left
     uint32_t* out = hist + pass * kSelBins;
     for (int i = threadIdx.x; i < kSelBins; i += kThreads)
         if (hist_s[i]) atomicAdd(&out[i], hist_s[i]);
+    publish_digit(status, hist, pass, prefix, want, scratch, result);
 }
 
 // Per tile: how many keys are above the threshold, how many equal it.
 __global__ void __launch_bounds__(kThreads)
-select_count_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, const uint32_t* hist,
-                    uint32_t* tile_counts) {
-    __shared__ uint32_t scratch[kThreads / 32 + 1];
-    __shared__ uint32_t result[2];
+select_count_kernel(const float* __restrict__ losses, int64_t N, const StatusBlock* status, uint32_t* tile_counts) {
     __shared__ uint32_t cnt[2];
-    uint32_t want;
-    const uint32_t T = resolve_prefix(hist, kSelPasses, k, want, scratch, result);
+    grid_dependency_wait();
+    const uint32_t T = __ldcg(&status->sel_prefix[kSelPasses - 1]);
     for (int64_t tile = blockIdx.x; tile * kTile < N; tile += gridDim.x) {
         if (threadIdx.x < 2) cnt[threadIdx.x] = 0;
         __syncthreads();
@@ -249,6 +287,7 @@ select_count_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, con
         __syncthreads();
         if (threadIdx.x < 2) tile_counts[2 * tile + threadIdx.x] = cnt[threadIdx.x];
         __syncthreads();
+        if (tile + gridDim.x >= (N + kTile - 1) / kTile) grid_launch_dependents();  // this CTA's last tile is done
     }
 }
 
@@ -258,22 +297,22 @@ select_count_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, con
 // (key, index) pairs for the sort and count their first sort digit.
 template <bool DIRECT>
 __global__ void __launch_bounds__(kThreads)
-select_emit_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, const uint32_t* hist,
-                   const uint32_t* __restrict__ tile_counts, int32_t* __restrict__ out_idx,
+select_emit_kernel(const float* __restrict__ losses, int64_t N, const StatusBlock* status,
+                   const uint32_t* tile_counts, int32_t* __restrict__ out_idx,
                    float* __restrict__ out_vals, uint32_t* __restrict__ out_keys, uint32_t* __restrict__ tile_hist) {
     __shared__ uint32_t scratch[kThreads / 32 + 1];
-    __shared__ uint32_t result[2];
     __shared__ uint32_t pre[2];
-    uint32_t r;
-    const uint32_t T = resolve_prefix(hist, kSelPasses, k, r, scratch, result);
+    grid_dependency_wait();
+    const uint32_t T = __ldcg(&status->sel_prefix[kSelPasses - 1]);
+    const uint32_t r = __ldcg(&status->sel_want[kSelPasses - 1]);
     for (int64_t tile = blockIdx.x; tile * kTile < N; tile += gridDim.x) {
         // entries above / equal to the threshold in the tiles before this one
         if (threadIdx.x < 2) pre[threadIdx.x] = 0;
         __syncthreads();
         uint32_t gt = 0, eq = 0;
         for (int64_t t = threadIdx.x; t < tile; t += kThreads) {
-            gt += tile_counts[2 * t];
-            eq += tile_counts[2 * t + 1];
+            gt += __ldcg(tile_counts + 2 * t);
+            eq += __ldcg(tile_counts + 2 * t + 1);
         }
         gt = warp_sum(static_cast<int>(gt));
         eq = warp_sum(static_cast<int>(eq));
@@ -287,6 +326,7 @@ select_emit_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, cons
         const int64_t base = tile * kTile + static_cast<int64_t>(threadIdx.x) * kPerThread;
         uint32_t key[kPerThread];
         load_keys(losses, N, base, key);
+        if (tile + gridDim.x >= (N + kTile - 1) / kTile) grid_launch_dependents();  // this CTA's last tile
         uint32_t my_gt = 0, my_eq = 0;
 #pragma unroll
         for (int i = 0; i < kPerThread; ++i) {
@@ -320,57 +360,101 @@ select_emit_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, cons
     }
 }
 
+// Lanes of the warp whose 8-bit digit equals this lane's, among the lanes with `live` set (0 for a lane that is
+// not live).  Nine votes; cheaper here than the generic match instruction.
+__device__ __forceinline__ uint32_t match_digit8(uint32_t d, bool live) {
+    uint32_t peers = __ballot_sync(0xFFFFFFFFu, live);
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+        const bool bit = (d >> b) & 1u;
+        const uint32_t m = __ballot_sync(0xFFFFFFFFu, bit);
+        peers &= bit ? m : ~m;
+    }
+    return live ? peers : 0u;
+}
+
 // One stable LSD pass over the selected pairs, on digit `pass` (8 bits, least
 // significant first), larger digits first.  Reads the digit counts per source
 // tile, ranks the tile's entries stably (warp match + per-warp counters), and
 // scatters.  Unless LAST, also counts the next digit per destination tile.
+// The pass is latency-bound (a short chain of dependent steps per tile), so a
+// tile is spread over 32 warps: four ranking rounds per warp instead of sixteen.
+constexpr int kSortThreads = 1024;
+
 template <bool LAST>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kSortThreads)
 sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restrict__ idx_in, uint32_t k, int pass,
                     const uint32_t* __restrict__ tile_hist, uint32_t* __restrict__ keys_out,
                     int32_t* __restrict__ idx_out, uint32_t* __restrict__ next_hist,
                     const float* __restrict__ losses, float* __restrict__ out_vals) {
-    constexpr int kWarps = kThreads / 32;
-    constexpr int kRounds = kTile / kThreads;  // 16 rounds of 32 consecutive entries per warp
+    constexpr int kWarps = kSortThreads / 32;
+    constexpr int kRounds = kTile / kSortThreads;  // rounds of 32 consecutive entries per warp
+    static_assert(kSortBins == 256 && kSortThreads >= kSortBins, "one thread per digit in the scans");
     __shared__ uint32_t counters[kWarps][kSortBins];
     __shared__ uint32_t base_s[kSortBins];
-    __shared__ uint32_t scratch[kThreads / 32 + 1];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __shared__ uint32_t tot_s[kSortBins];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t tiles = (k + kTile - 1) / kTile;
     const int shift = 8 * pass;
+    grid_dependency_wait();
     for (uint32_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
         // where each digit's run starts for this tile: all entries of earlier digits, plus
         // this digit's entries in earlier tiles
-        {
-            const int d = threadIdx.x;  // kThreads == kSortBins
-            uint32_t total = 0, before = 0;
-            for (uint32_t t = 0; t < tiles; ++t) {
-                const uint32_t c = tile_hist[t * kSortBins + d];
-                total += c;
-                before += t < tile ? c : 0u;
-            }
-            const uint32_t excl = block_exclusive_scan(total, scratch);
-            base_s[d] = excl + before;
+        uint32_t before = 0;
+        if (tid < kSortBins) {
+            uint32_t total = 0;
+            for (uint32_t t0 = 0; t0 < tiles; t0 += 8) {
+                uint32_t c[8];
 #pragma unroll
-            for (int w = 0; w < kWarps; ++w) counters[w][d] = 0;
+                for (int u = 0; u < 8; ++u)  // eight independent loads in flight
+                    c[u] = t0 + u < tiles ? __ldcg(tile_hist + (t0 + u) * kSortBins + tid) : 0u;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    total += c[u];
+                    before += t0 + u < tile ? c[u] : 0u;
+                }
+            }
+            tot_s[tid] = total;
         }
-        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < kWarps * kSortBins / kSortThreads; ++i) (&counters[0][0])[i * kSortThreads + tid] = 0;
         uint32_t key[kRounds], rank[kRounds];
         int32_t idx[kRounds];
         const uint32_t first = tile * kTile + warp * (kRounds * 32);
 #pragma unroll
         for (int rd = 0; rd < kRounds; ++rd) {  // all loads first: they are independent
             const uint32_t e = first + rd * 32 + lane;
-            key[rd] = e < k ? keys_in[e] : 0u;
-            idx[rd] = e < k ? idx_in[e] : 0;
+            key[rd] = e < k ? __ldcg(keys_in + e) : 0u;
+            idx[rd] = e < k ? __ldcg(idx_in + e) : 0;
+        }
+        __syncthreads();
+        if (warp == 0) {  // exclusive scan of the 256 digit totals, eight per lane
+            uint32_t v[8], sum = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                v[i] = tot_s[lane * 8 + i];
+                sum += v[i];
+            }
+            uint32_t inc = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                if (lane >= o) inc += n;
+            }
+            uint32_t run = inc - sum;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                tot_s[lane * 8 + i] = run;
+                run += v[i];
+            }
         }
 #pragma unroll
         for (int rd = 0; rd < kRounds; ++rd) {
             const uint32_t e = first + rd * 32 + lane;
             const bool live = e < k;
-            const uint32_t dd = live ? 255u - ((key[rd] >> shift) & 0xFFu) : 256u;
-            const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dd);
-            const int leader = __ffs(peers) - 1;
+            const uint32_t dd = 255u - ((key[rd] >> shift) & 0xFFu);
+            const uint32_t peers = match_digit8(dd, live);
+            const int leader = live ? __ffs(peers) - 1 : lane;
             uint32_t old = 0;
             if (live && lane == leader) {
                 old = counters[warp][dd];
@@ -381,29 +465,45 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
             __syncwarp();
         }
         __syncthreads();
-        {
-            const int d = threadIdx.x;
+        if (tid < kSortBins) {
+            base_s[tid] = tot_s[tid] + before;
             uint32_t run = 0;
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) {
-                const uint32_t c = counters[w][d];
-                counters[w][d] = run;
+                const uint32_t c = counters[w][tid];
+                counters[w][tid] = run;
                 run += c;
             }
         }
         __syncthreads();
+        if (tile + gridDim.x >= tiles) grid_launch_dependents();  // only this CTA's last scatter is left
 #pragma unroll
         for (int rd = 0; rd < kRounds; ++rd) {
             const uint32_t e = first + rd * 32 + lane;
-            if (e < k) {
+            const bool live = e < k;
+            uint32_t pos = 0;
+            if (live) {
                 const uint32_t dd = 255u - ((key[rd] >> shift) & 0xFFu);
-                const uint32_t pos = base_s[dd] + counters[warp][dd] + rank[rd];
+                pos = base_s[dd] + counters[warp][dd] + rank[rd];
                 idx_out[pos] = idx[rd];
                 if (LAST) {
                     if (out_vals) out_vals[pos] = losses[idx[rd]];
                 } else {
                     keys_out[pos] = key[rd];
-                    atomicAdd(&next_hist[(pos / kTile) * kSortBins + (255u - ((key[rd] >> (shift + 8)) & 0xFFu))], 1u);
+                }
+            }
+            if (!LAST) {
+                // count the next digit per destination tile.  High digits are nearly constant over the selection,
+                // so a warp sends one atomic per distinct counter instead of one per entry.
+                const uint32_t nd = 255u - ((key[rd] >> (shift + 8)) & 0xFFu);
+                const uint32_t peers = match_digit8(nd, live);
+                const int leader = live ? __ffs(peers) - 1 : lane;
+                const uint32_t t = pos / kTile;
+                const bool with_leader = t == __shfl_sync(0xFFFFFFFFu, t, leader);  // same destination tile as the leader
+                const uint32_t same = __ballot_sync(0xFFFFFFFFu, live && with_leader);
+                if (live) {
+                    if (lane == leader) atomicAdd(&next_hist[t * kSortBins + nd], static_cast<uint32_t>(__popc(peers & same)));
+                    else if (!with_leader) atomicAdd(&next_hist[t * kSortBins + nd], 1u);
                 }
             }
         }
@@ -420,6 +520,7 @@ small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int
                   float* __restrict__ out_vals) {
     __shared__ unsigned long long ck[kSmallN];
     __shared__ uint32_t warp_tot[kSmallThreads / 32];
+    grid_dependency_wait();
     int n2 = 1;
     while (n2 < n) n2 <<= 1;
     for (int i = threadIdx.x; i < n2; i += kSmallThreads)
@@ -440,6 +541,7 @@ small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int
             }
             __syncthreads();
         }
+    grid_launch_dependents();
     if (order == LSGD_ORDER_LOSS_DESC) {
         for (int j = threadIdx.x; j < k; j += kSmallThreads) {
             const int32_t i = static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(ck[j]));
@@ -484,35 +586,34 @@ small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int
 
 cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order order, int32_t* out_idx,
                         float* out_vals, const TopkWorkspace& ws, bool hist0_ready, cudaStream_t s) {
-    if (N <= kSmallN) {
-        small_topk_kernel<<<1, kSmallThreads, 0, s>>>(losses, static_cast<int>(N), static_cast<int>(k),
-                                                      static_cast<int>(order), out_idx, out_vals);
-        return cudaGetLastError();
-    }
+    if (N <= kSmallN)
+        return launch_dependent(small_topk_kernel, 1, kSmallThreads, s, losses, static_cast<int>(N), static_cast<int>(k),
+                                static_cast<int>(order), out_idx, out_vals);
     const int64_t tiles_n = (N + kTile - 1) / kTile;
     const int grid_n = static_cast<int>(std::min<int64_t>(tiles_n, static_cast<int64_t>(sm_count()) * 8));
     const uint32_t kk = static_cast<uint32_t>(k);
-    for (int pass = hist0_ready ? 1 : 0; pass < kSelPasses; ++pass)
-        select_hist_kernel<<<grid_n, kThreads, 0, s>>>(losses, N, kk, pass, ws.hist);
-    select_count_kernel<<<grid_n, kThreads, 0, s>>>(losses, N, kk, ws.hist, ws.tile_counts);
-    if (order == LSGD_ORDER_INDEX_ASC) {
-        select_emit_kernel<true><<<grid_n, kThreads, 0, s>>>(losses, N, kk, ws.hist, ws.tile_counts, out_idx, out_vals,
-                                                             nullptr, nullptr);
-        return cudaGetLastError();
-    }
+    cudaError_t e = cudaSuccess;
+    for (int pass = hist0_ready ? 1 : 0; pass < kSelPasses && e == cudaSuccess; ++pass)
+        e = launch_dependent(select_hist_kernel, grid_n, kThreads, s, losses, N, kk, pass,
+                             pass > (hist0_ready ? 1 : 0), ws.hist, ws.status);
+    if (e != cudaSuccess) return e;
+    e = launch_dependent(select_count_kernel, grid_n, kThreads, s, losses, N, ws.status, ws.tile_counts);
+    if (e != cudaSuccess) return e;
+    if (order == LSGD_ORDER_INDEX_ASC)
+        return launch_dependent(select_emit_kernel<true>, grid_n, kThreads, s, losses, N, ws.status, ws.tile_counts,
+                                out_idx, out_vals, nullptr, nullptr);
     const int64_t tiles_k = (k + kTile - 1) / kTile;
     const size_t th = static_cast<size_t>(tiles_k) * kSortBins;
-    select_emit_kernel<false><<<grid_n, kThreads, 0, s>>>(losses, N, kk, ws.hist, ws.tile_counts, ws.idx[0], nullptr,
-                                                          ws.keys[0], ws.tile_hist);
-    const int grid_k = static_cast<int>(std::min<int64_t>(tiles_k, static_cast<int64_t>(sm_count()) * 4));
-    for (int pass = 0; pass < 3; ++pass)
-        sort_scatter_kernel<false><<<grid_k, kThreads, 0, s>>>(ws.keys[pass & 1], ws.idx[pass & 1], kk, pass,
-                                                               ws.tile_hist + pass * th, ws.keys[(pass + 1) & 1],
-                                                               ws.idx[(pass + 1) & 1], ws.tile_hist + (pass + 1) * th,
-                                                               nullptr, nullptr);
-    sort_scatter_kernel<true><<<grid_k, kThreads, 0, s>>>(ws.keys[1], ws.idx[1], kk, 3, ws.tile_hist + 3 * th, nullptr,
-                                                          out_idx, nullptr, losses, out_vals);
-    return cudaGetLastError();
+    e = launch_dependent(select_emit_kernel<false>, grid_n, kThreads, s, losses, N, ws.status, ws.tile_counts, ws.idx[0],
+                         nullptr, ws.keys[0], ws.tile_hist);
+    const int grid_k = static_cast<int>(std::min<int64_t>(tiles_k, static_cast<int64_t>(sm_count()) * 2));
+    for (int pass = 0; pass < 3 && e == cudaSuccess; ++pass)
+        e = launch_dependent(sort_scatter_kernel<false>, grid_k, kSortThreads, s, ws.keys[pass & 1], ws.idx[pass & 1], kk, pass,
+                             ws.tile_hist + pass * th, ws.keys[(pass + 1) & 1], ws.idx[(pass + 1) & 1],
+                             ws.tile_hist + (pass + 1) * th, nullptr, nullptr);
+    if (e != cudaSuccess) return e;
+    return launch_dependent(sort_scatter_kernel<true>, grid_k, kSortThreads, s, ws.keys[1], ws.idx[1], kk, 3,
+                            ws.tile_hist + 3 * th, nullptr, out_idx, nullptr, losses, out_vals);
 }
 
 }  // namespace lsgd
