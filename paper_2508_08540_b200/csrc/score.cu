@@ -13,14 +13,16 @@
 // whose argument equals (x_j - m) L + d with d = fma(m, L, -fl(m L)) known
 // exactly; the common factor 2^d is divided out once per row.
 //
-// Three row shapes, three kernels (all bound by the bytes of the logits):
+// Row shapes and their kernels (all bound by the bytes of the logits):
 //   tiny rows   (C <= 32)         one thread per row out of a shared-memory tile
+//   small rows  (C <= 256)        4 or 8 lanes per row out of a shared-memory tile
 //   short rows  (<= 4064 bytes)   one warp per row, the row held in registers
 //   long rows   (<= 256 KB)       a ring of 4 KB chunk buffers per SM filled by bulk
 //                                 asynchronous copies (TMA, 1-D); free-running warps
 //                                 reduce chunks to (max, sum) records
 //   anything longer               one CTA per row, two passes over global memory
-// Rows whose label is ignore_index are never read.
+// Rows whose label is ignore_index are never scored; the kernels for short, long and longer rows do not even
+// read them (tiny and small rows are copied tile-wise, ignored rows included).
 #include <cuda_bf16.h>
 
 #include <algorithm>
@@ -152,6 +154,173 @@ score_tiny_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
             h.add(loss);
         }
     }
+    __syncthreads();
+    h.flush();
+}
+
+// ---------------------------------------------------------------------------
+// Small rows (32 < C <= 256): a CTA copies a tile of consecutive rows (one
+// contiguous, 16-byte-aligned-superset byte range) into shared memory with
+// vector loads; groups of L lanes then own one row each and read it from there.
+// One warp per row would spend most of its instructions on 32-lane reductions
+// and on the per-row epilogue; with L lanes per row those are shared by 32 / L
+// rows.  VEC: every row starts on a 16-byte boundary (base aligned, row bytes a
+// multiple of 16), so a lane reads 16-byte chunks l, l + L, ... of its row;
+// otherwise it reads elements l, l + L, ...
+// ---------------------------------------------------------------------------
+constexpr int kGroupThreads = 256;
+constexpr int kGroupMaxC = 256;
+constexpr int kGroupStages = 3;
+
+template <typename T>
+__device__ __forceinline__ void unpack_chunk(const uint4& q, float (&v)[Elem<T>::kPerVec]) {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+    if constexpr (Elem<T>::kPerVec == 4) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = __uint_as_float(w[e]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {  // bf16 is the upper half of an fp32
+            v[2 * e] = __uint_as_float(w[e] << 16);
+            v[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
+        }
+    }
+}
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst))),
+                 "l"(gsrc)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
+}
+
+// Tiles flow through a ring of kGroupStages buffers filled by asynchronous 16-byte copies (global -> shared, past
+// the registers), two tiles ahead of the one being reduced, so every CTA always has loads in flight.
+template <typename T, int L, bool VEC>
+__global__ void __launch_bounds__(kGroupThreads)
+score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
+                        int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0,
+                        int stage_bytes) {
+    constexpr int R = kGroupThreads / L;  // rows per tile = lane groups per CTA
+    constexpr int EPV = Elem<T>::kPerVec;
+    extern __shared__ __align__(16) unsigned char group_smem[];
+    uint32_t* hist_s = reinterpret_cast<uint32_t*>(group_smem);
+    unsigned char* stages = group_smem + kSelBins * sizeof(uint32_t);
+    Hist0 h{hist_s, hist0};
+    h.clear();
+    const int row_bytes = C * static_cast<int>(sizeof(T));
+    const int64_t tiles = (rows + R - 1) / R;
+    const int g = threadIdx.x / L, l = threadIdx.x % L;
+    // VEC, L == 4: two rows share a quarter-warp's 16-byte accesses, so rows are laid out in shared memory with
+    // a pitch of 4 (mod 8) chunks, which puts neighbouring rows four bank groups apart whatever the row length.
+    // (The order in which a row's elements are summed must not depend on where the row sits: copies of a row
+    // have to score the same bits.)
+    const int nchunk = row_bytes >> 4;
+    const int pitch16 = (VEC && L == 4) ? nchunk + ((4 - nchunk) & 7) : nchunk;
+    const float inv_nchunk = 1.0f / static_cast<float>(nchunk > 0 ? nchunk : 1);
+    const int64_t my_tiles = tiles > blockIdx.x ? (tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+    auto issue = [&](int64_t i) {  // requests this CTA's i-th tile into stage i % kGroupStages
+        if (i < my_tiles) {
+            const int64_t row0 = (blockIdx.x + i * gridDim.x) * R;
+            const int nrows = rows - row0 < R ? static_cast<int>(rows - row0) : R;
+            const uintptr_t b0 = reinterpret_cast<uintptr_t>(logits) + row0 * row_bytes;
+            const int head = VEC ? 0 : static_cast<int>(b0 & 15);
+            const uint4* src = reinterpret_cast<const uint4*>(b0 - head);
+            const int nvec = (head + nrows * row_bytes + 15) >> 4;  // an aligned block that holds a valid byte is safe to read
+            uint4* dst = reinterpret_cast<uint4*>(stages + (i % kGroupStages) * stage_bytes);
+            for (int v = threadIdx.x; v < nvec; v += kGroupThreads) {
+                int d = v;
+                if constexpr (VEC && L == 4) {
+                    const int r = __float2int_rz((static_cast<float>(v) + 0.5f) * inv_nchunk);  // v / nchunk, exact here
+                    d = r * pitch16 + (v - r * nchunk);
+                }
+                cp_async16(dst + d, src + v);
+            }
+        }
+        cp_async_commit();  // one group per tile slot, also when it is empty: the wait below counts groups
+    };
+    auto label_of = [&](int64_t i) -> int64_t {
+        if (i >= my_tiles) return ignore_index;
+        const int64_t row = (blockIdx.x + i * gridDim.x) * R + g;
+        return row < rows ? labels[row] : ignore_index;
+    };
+
+#pragma unroll
+    for (int i = 0; i < kGroupStages - 1; ++i) issue(i);
+    int64_t y = label_of(0);
+    for (int64_t i = 0; i < my_tiles; ++i) {
+        issue(i + kGroupStages - 1);
+        const int64_t y_next = label_of(i + 1);
+        cp_async_wait<kGroupStages - 1>();
+        __syncthreads();  // everybody's copies of tile i have landed
+        const int64_t row0 = (blockIdx.x + i * gridDim.x) * R;
+        const bool mine = row0 + g < rows;
+        const int head = VEC ? 0 : static_cast<int>((reinterpret_cast<uintptr_t>(logits) + row0 * row_bytes) & 15);
+        const unsigned char* buf = stages + (i % kGroupStages) * stage_bytes;
+        const int cls = mine ? label_class(y, C, ignore_index) : 1;
+        const T* x = reinterpret_cast<const T*>(buf + head + g * (VEC ? pitch16 * 16 : row_bytes));
+        float m = neg_inf(), s = 0.f;
+        int n_max = 0;
+        if constexpr (VEC) {
+            const uint4* xv = reinterpret_cast<const uint4*>(x);
+            const int nch = cls == 0 ? nchunk : 0;  // groups without a row to score run the reductions on nothing
+#pragma unroll 2
+            for (int c = l; c < nch; c += L) {
+                float v[EPV];
+                unpack_chunk<T>(xv[c], v);
+#pragma unroll
+                for (int e = 0; e < EPV; ++e) m = fmaxf(m, v[e]);
+            }
+#pragma unroll
+            for (int o = L / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+            const RowScale rs(m);
+#pragma unroll 2
+            for (int c = l; c < nch; c += L) {
+                float v[EPV];
+                unpack_chunk<T>(xv[c], v);
+#pragma unroll
+                for (int e = 0; e < EPV; ++e) {
+                    if (v[e] < m) s += ex2(fmaf(v[e], kLog2e, rs.nml));
+                    else ++n_max;
+                }
+            }
+        } else {
+            const int n = cls == 0 ? C : 0;
+            for (int j = l; j < n; j += L) m = fmaxf(m, Elem<T>::widen(x[j]));
+#pragma unroll
+            for (int o = L / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+            const RowScale rs(m);
+            for (int j = l; j < n; j += L) {
+                const float v = Elem<T>::widen(x[j]);
+                if (v < m) s += ex2(fmaf(v, kLog2e, rs.nml));
+                else ++n_max;
+            }
+        }
+#pragma unroll
+        for (int o = L / 2; o > 0; o >>= 1) {
+            s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+            n_max += __shfl_xor_sync(0xFFFFFFFFu, n_max, o);
+        }
+        if (mine && l == 0) {
+            float loss = 0.f;
+            if (cls == 2) {
+                loss = __uint_as_float(0x7FC00000u);
+                atomicAdd(&status->bad_labels, 1);
+            } else if (cls == 0) {
+                loss = finish_loss(m, Elem<T>::widen(x[static_cast<int>(y)]), s, n_max, RowScale(m));
+            }
+            row_loss[row0 + g] = loss;
+            h.add(loss);
+        }
+        __syncthreads();  // the stage may be refilled
+        y = y_next;
+    }
+    cp_async_wait<0>();
     __syncthreads();
     h.flush();
 }
@@ -798,6 +967,30 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
         score_tiny_rows_kernel<T><<<grid, kTinyThreads, 0, s>>>(logits, labels, rows, static_cast<int>(C),
                                                                  ignore_index, row_loss, status, hist0);
         return cudaGetLastError();
+    }
+    if (C <= kGroupMaxC) {
+        const bool vec = (reinterpret_cast<uintptr_t>(logits) & 15) == 0 && row_bytes % 16 == 0;
+        cudaError_t err = cudaSuccess;
+        auto go = [&](auto kernel, int lanes) {
+            const int tile_rows = kGroupThreads / lanes;
+            // bytes of one stage: the rows of a tile at their shared-memory pitch (rows of 16-byte chunks handled by
+            // 4 lanes are padded to 4 (mod 8) chunks), or the flat copy of the tile's aligned superset
+            const int64_t nchunk = row_bytes / 16;
+            const int64_t pitch = vec ? 16 * (lanes == 4 ? nchunk + ((4 - nchunk) & 7) : nchunk) : row_bytes;
+            const int stage_bytes = static_cast<int>((tile_rows * pitch + 32 + 15) / 16 * 16);
+            const size_t smem = kSelBins * sizeof(uint32_t) + static_cast<size_t>(kGroupStages) * stage_bytes;
+            err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynSmem));
+            if (err != cudaSuccess) return;
+            const int64_t tiles = (rows + tile_rows - 1) / tile_rows;
+            const int grid = static_cast<int>(std::min<int64_t>(tiles, static_cast<int64_t>(sms) * blocks_per_sm(kernel, kGroupThreads, smem)));
+            kernel<<<grid, kGroupThreads, smem, s>>>(logits, labels, rows, static_cast<int>(C), ignore_index, row_loss,
+                                                     status, hist0, stage_bytes);
+            err = cudaGetLastError();
+        };
+        // rows per tile (256 / L) times bytes per row (<= 4 C): at most 64 x 512 or 32 x 1024 bytes per stage, plus padding
+        if (C <= 128) vec ? go(score_group_rows_kernel<T, 4, true>, 4) : go(score_group_rows_kernel<T, 4, false>, 4);
+        else vec ? go(score_group_rows_kernel<T, 8, true>, 8) : go(score_group_rows_kernel<T, 8, false>, 8);
+        return err;
     }
     const int64_t need_vec = (row_bytes + 30) / 16;  // vectors of the aligned superset, worst alignment
     if (need_vec <= 256) {

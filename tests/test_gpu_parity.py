@@ -51,7 +51,11 @@ SCORE_SHAPES = [
     # N, T, C, dtype            path
     (1, 1, 1, "f32"), (33, 1, 2, "f32"), (1000, 1, 3, "f32"), (777, 1, 7, "bf16"), (5000, 1, 10, "f32"),
     (300, 1, 32, "bf16"),                                                        # tiny rows
-    (31, 1, 33, "f32"), (2049, 1, 100, "f32"), (513, 1, 100, "bf16"), (257, 1, 1000, "f32"),
+    (31, 1, 33, "f32"), (2049, 1, 100, "f32"), (513, 1, 100, "bf16"),
+    (1000, 1, 36, "f32"), (333, 2, 40, "bf16"), (4099, 1, 64, "f32"), (777, 1, 102, "f32"), (650, 1, 128, "bf16"),
+    (129, 3, 128, "f32"), (1031, 1, 132, "f32"), (500, 1, 200, "f32"), (97, 2, 201, "f32"), (420, 1, 256, "f32"),
+    (801, 1, 256, "bf16"), (65, 1, 255, "bf16"),                                 # lane groups: 16-byte rows or not, 4 / 8 lanes
+    (257, 1, 1000, "f32"),
     (65, 3, 1016, "f32"), (40, 2, 2031, "bf16"), (129, 1, 999, "bf16"),          # warp rows, odd alignments
     (37, 1, 1017, "f32"), (19, 2, 2500, "f32"), (24, 3, 4099, "bf16"), (6, 5, 30522, "bf16"),
     (5, 1, 50001, "f32"),                                                        # CTA rows (shared-memory resident)
