@@ -92,7 +92,7 @@ LSGD_API size_t lsgd_score_topk_workspace_bytes(int64_t N, int64_t T, int64_t C,
  *   logits  device, [N, T, C] row-major, contiguous, dtype `dtype`, aligned to
  *           its element size (16-byte alignment is faster, not required).
  *           Values must be finite.  Rows whose label is ignore_index are not scored,
- *           and rows longer than 1 KB are then not read at all (shorter rows are
+ *           and rows longer than 2 KB are then not read at all (shorter rows are
  *           loaded in contiguous tiles, ignored rows included; their values are
  *           not used).
  *   labels  device, [N, T] int64.  A label outside [0, C) that is not

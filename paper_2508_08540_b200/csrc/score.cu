@@ -15,7 +15,7 @@
 //
 // Row shapes and their kernels (all bound by the bytes of the logits):
 //   tiny rows   (C <= 32)         one thread per row out of a shared-memory tile
-//   small rows  (C <= 256)        4 or 8 lanes per row out of a shared-memory tile
+//   small rows  (<= 2 KB)         4, 8 or 16 lanes per row out of a shared-memory tile
 //   short rows  (<= 4064 bytes)   one warp per row, the row held in registers
 //   long rows   (<= 256 KB)       a ring of 4 KB chunk buffers per SM filled by bulk
 //                                 asynchronous copies (TMA, 1-D); free-running warps
@@ -26,6 +26,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <type_traits>
 
 #include "lsgd_internal.cuh"
 
@@ -159,28 +160,41 @@ score_tiny_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
 }
 
 // ---------------------------------------------------------------------------
-// Small rows (32 < C <= 256): a CTA copies a tile of consecutive rows (one
+// Small rows (C > 32, at most 2 KB): a CTA copies a tile of consecutive rows (one
 // contiguous, 16-byte-aligned-superset byte range) into shared memory with
 // vector loads; groups of L lanes then own one row each and read it from there.
 // One warp per row would spend most of its instructions on 32-lane reductions
 // and on the per-row epilogue; with L lanes per row those are shared by 32 / L
-// rows.  VEC: every row starts on a 16-byte boundary (base aligned, row bytes a
-// multiple of 16), so a lane reads 16-byte chunks l, l + L, ... of its row;
-// otherwise it reads elements l, l + L, ...
+// rows.  With a 16-byte-aligned base, rows start on 16-, 8- or 4-byte boundaries
+// according to their length, and a lane reads chunks of that size, l, l + L, ...
+// of its row; otherwise it reads elements l, l + L, ...
 // ---------------------------------------------------------------------------
 constexpr int kGroupThreads = 256;
-constexpr int kGroupMaxC = 256;
+constexpr int kGroupMaxRowBytes = 2048;
 constexpr int kGroupStages = 2;
 
-template <typename T>
-__device__ __forceinline__ void unpack_chunk(const uint4& q, float (&v)[Elem<T>::kPerVec]) {
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-    if constexpr (Elem<T>::kPerVec == 4) {
+// A chunk: the CB bytes (16, 8 or 4) a lane reads from shared memory at once, CB / sizeof(T) elements.
+template <int CB>
+struct ChunkWord;
+template <>
+struct ChunkWord<16> { using type = uint4; };
+template <>
+struct ChunkWord<8> { using type = uint2; };
+template <>
+struct ChunkWord<4> { using type = uint32_t; };
+
+template <typename T, int CB>
+__device__ __forceinline__ void unpack_chunk(const typename ChunkWord<CB>::type& q, float (&v)[CB / static_cast<int>(sizeof(T))]) {
+    uint32_t w[CB / 4];
+    if constexpr (CB == 16) { w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w; }
+    else if constexpr (CB == 8) { w[0] = q.x; w[1] = q.y; }
+    else { w[0] = q; }
+    if constexpr (sizeof(T) == 4) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) v[e] = __uint_as_float(w[e]);
+        for (int e = 0; e < CB / 4; ++e) v[e] = __uint_as_float(w[e]);
     } else {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {  // bf16 is the upper half of an fp32
+        for (int e = 0; e < CB / 4; ++e) {  // bf16 is the upper half of an fp32
             v[2 * e] = __uint_as_float(w[e] << 16);
             v[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
         }
@@ -201,13 +215,15 @@ __device__ __forceinline__ void cp_async_wait() {
 // Tiles flow through a ring of kGroupStages buffers filled by asynchronous 16-byte copies (global -> shared, past
 // the registers), one tile ahead of the one being reduced, so every CTA always has loads in flight; two stages
 // rather than three leave room for a third CTA per SM, which is worth more (measured).
-template <typename T, int L, bool VEC>
+template <typename T, int L, int CB>
 __global__ void __launch_bounds__(kGroupThreads)
 score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
                         int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0,
                         int stage_bytes) {
     constexpr int R = kGroupThreads / L;  // rows per tile = lane groups per CTA
-    constexpr int EPV = Elem<T>::kPerVec;
+    constexpr bool VEC = CB > 0;          // rows start on CB-byte boundaries and are whole chunks (base 16-byte aligned)
+    constexpr bool PADDED = CB == 16 && L < 8;
+    constexpr int EPV = VEC ? CB / static_cast<int>(sizeof(T)) : 1;
     extern __shared__ __align__(16) unsigned char group_smem[];
     uint32_t* hist_s = reinterpret_cast<uint32_t*>(group_smem);
     unsigned char* stages = group_smem + kSelBins * sizeof(uint32_t);
@@ -216,12 +232,12 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
     const int row_bytes = C * static_cast<int>(sizeof(T));
     const int64_t tiles = (rows + R - 1) / R;
     const int g = threadIdx.x / L, l = threadIdx.x % L;
-    // VEC, L == 4: two rows share a quarter-warp's 16-byte accesses, so rows are laid out in shared memory with
+    // 16-byte chunks, L == 4: two rows share a quarter-warp's accesses, so rows are laid out in shared memory with
     // a pitch of 4 (mod 8) chunks, which puts neighbouring rows four bank groups apart whatever the row length.
     // (The order in which a row's elements are summed must not depend on where the row sits: copies of a row
     // have to score the same bits.)
-    const int nchunk = row_bytes >> 4;
-    const int pitch16 = (VEC && L == 4) ? nchunk + ((4 - nchunk) & 7) : nchunk;
+    const int nchunk = VEC ? row_bytes / (VEC ? CB : 1) : 0;
+    const int pitch_bytes = PADDED ? 16 * (nchunk + ((L - nchunk) & 7)) : row_bytes;
     const float inv_nchunk = 1.0f / static_cast<float>(nchunk > 0 ? nchunk : 1);
     const int64_t my_tiles = tiles > blockIdx.x ? (tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
@@ -236,9 +252,9 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
             uint4* dst = reinterpret_cast<uint4*>(stages + (i % kGroupStages) * stage_bytes);
             for (int v = threadIdx.x; v < nvec; v += kGroupThreads) {
                 int d = v;
-                if constexpr (VEC && L == 4) {
+                if constexpr (PADDED) {
                     const int r = __float2int_rz((static_cast<float>(v) + 0.5f) * inv_nchunk);  // v / nchunk, exact here
-                    d = r * pitch16 + (v - r * nchunk);
+                    d = r * (pitch_bytes >> 4) + (v - r * nchunk);
                 }
                 cp_async16(dst + d, src + v);
             }
@@ -264,16 +280,17 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
         const int head = VEC ? 0 : static_cast<int>((reinterpret_cast<uintptr_t>(logits) + row0 * row_bytes) & 15);
         const unsigned char* buf = stages + (i % kGroupStages) * stage_bytes;
         const int cls = mine ? label_class(y, C, ignore_index) : 1;
-        const T* x = reinterpret_cast<const T*>(buf + head + g * (VEC ? pitch16 * 16 : row_bytes));
+        const T* x = reinterpret_cast<const T*>(buf + head + g * pitch_bytes);
         float m = neg_inf(), s = 0.f;
         int n_max = 0;
         if constexpr (VEC) {
-            const uint4* xv = reinterpret_cast<const uint4*>(x);
+            using Word = typename ChunkWord<VEC ? CB : 16>::type;
+            const Word* xv = reinterpret_cast<const Word*>(x);
             const int nch = cls == 0 ? nchunk : 0;  // groups without a row to score run the reductions on nothing
 #pragma unroll 2
             for (int c = l; c < nch; c += L) {
                 float v[EPV];
-                unpack_chunk<T>(xv[c], v);
+                unpack_chunk<T, VEC ? CB : 16>(xv[c], v);
 #pragma unroll
                 for (int e = 0; e < EPV; ++e) m = fmaxf(m, v[e]);
             }
@@ -283,7 +300,7 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
 #pragma unroll 2
             for (int c = l; c < nch; c += L) {
                 float v[EPV];
-                unpack_chunk<T>(xv[c], v);
+                unpack_chunk<T, VEC ? CB : 16>(xv[c], v);
 #pragma unroll
                 for (int e = 0; e < EPV; ++e) {
                     if (v[e] < m) s += ex2(fmaf(v[e], kLog2e, rs.nml));
@@ -969,15 +986,16 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
                                                                  ignore_index, row_loss, status, hist0);
         return cudaGetLastError();
     }
-    if (C <= kGroupMaxC) {
-        const bool vec = (reinterpret_cast<uintptr_t>(logits) & 15) == 0 && row_bytes % 16 == 0;
+    if (row_bytes <= kGroupMaxRowBytes) {
+        const bool base_ok = (reinterpret_cast<uintptr_t>(logits) & 15) == 0;
+        const int cb = !base_ok ? 0 : row_bytes % 16 == 0 ? 16 : row_bytes % 8 == 0 ? 8 : row_bytes % 4 == 0 ? 4 : 0;
         cudaError_t err = cudaSuccess;
         auto go = [&](auto kernel, int lanes) {
             const int tile_rows = kGroupThreads / lanes;
             // bytes of one stage: the rows of a tile at their shared-memory pitch (rows of 16-byte chunks handled by
             // 4 lanes are padded to 4 (mod 8) chunks), or the flat copy of the tile's aligned superset
             const int64_t nchunk = row_bytes / 16;
-            const int64_t pitch = vec ? 16 * (lanes == 4 ? nchunk + ((4 - nchunk) & 7) : nchunk) : row_bytes;
+            const int64_t pitch = (cb == 16 && lanes < 8) ? 16 * (nchunk + ((lanes - nchunk) & 7)) : row_bytes;
             const int stage_bytes = static_cast<int>((tile_rows * pitch + 32 + 15) / 16 * 16);
             const size_t smem = kSelBins * sizeof(uint32_t) + static_cast<size_t>(kGroupStages) * stage_bytes;
             err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynSmem));
@@ -988,9 +1006,17 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
                                                      status, hist0, stage_bytes);
             err = cudaGetLastError();
         };
-        // rows per tile (256 / L) times bytes per row (<= 4 C): at most 64 x 512 or 32 x 1024 bytes per stage, plus padding
-        if (C <= 128) vec ? go(score_group_rows_kernel<T, 4, true>, 4) : go(score_group_rows_kernel<T, 4, false>, 4);
-        else vec ? go(score_group_rows_kernel<T, 8, true>, 8) : go(score_group_rows_kernel<T, 8, false>, 8);
+        auto by_chunk = [&](auto lanes_tag) {
+            constexpr int LN = decltype(lanes_tag)::value;
+            if (cb == 16) go(score_group_rows_kernel<T, LN, 16>, LN);
+            else if (cb == 8) go(score_group_rows_kernel<T, LN, 8>, LN);
+            else if (cb == 4 && sizeof(T) == 2) go(score_group_rows_kernel<T, LN, 4>, LN);
+            else go(score_group_rows_kernel<T, LN, 0>, LN);  // (4-byte chunks of fp32 are single elements)
+        };
+        // rows per tile (256 / L) times bytes per row: at most 32 KB per stage (64 x 512, 32 x 1024, 16 x 2048), plus padding
+        if (row_bytes <= 512) by_chunk(std::integral_constant<int, 4>{});
+        else if (row_bytes <= 1024) by_chunk(std::integral_constant<int, 8>{});
+        else by_chunk(std::integral_constant<int, 16>{});
         return err;
     }
     const int64_t need_vec = (row_bytes + 30) / 16;  // vectors of the aligned superset, worst alignment

@@ -54,7 +54,9 @@ SCORE_SHAPES = [
     (31, 1, 33, "f32"), (2049, 1, 100, "f32"), (513, 1, 100, "bf16"),
     (1000, 1, 36, "f32"), (333, 2, 40, "bf16"), (4099, 1, 64, "f32"), (777, 1, 102, "f32"), (650, 1, 128, "bf16"),
     (129, 3, 128, "f32"), (1031, 1, 132, "f32"), (500, 1, 200, "f32"), (97, 2, 201, "f32"), (420, 1, 256, "f32"),
-    (801, 1, 256, "bf16"), (65, 1, 255, "bf16"),                                 # lane groups: 16-byte rows or not, 4 / 8 lanes
+    (801, 1, 256, "bf16"), (65, 1, 255, "bf16"), (900, 1, 102, "bf16"), (211, 1, 300, "f32"), (150, 2, 512, "f32"),
+    (300, 1, 1000, "bf16"), (77, 3, 1024, "bf16"), (190, 1, 450, "bf16"), (100, 1, 511, "f32"),
+                                                                                 # lane groups: 16/8/4-byte rows or not, 4/8/16 lanes
     (257, 1, 1000, "f32"),
     (65, 3, 1016, "f32"), (40, 2, 2031, "bf16"), (129, 1, 999, "bf16"),          # warp rows, odd alignments
     (37, 1, 1017, "f32"), (19, 2, 2500, "f32"), (24, 3, 4099, "bf16"), (6, 5, 30522, "bf16"),
