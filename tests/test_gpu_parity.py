@@ -1,6 +1,6 @@
 """Element-by-element parity of the CUDA library (through its C ABI) with the CPU
 oracle on the same seeded inputs: small and ragged shapes, several tiles, edge
-cases.  Tolerances (stated here, derived in the design doc):
+cases.  Tolerances (from the arithmetic: 2-ulp exponentials and a tree sum for the losses, a chain of P fused multiply-adds for Eq. 3):
   losses       |g - o| <= 1e-5 |o| + C 2^-52   (C 2^-52: the oracle's own double rounding when it sums C terms next to 1;
                losses below that floor are checked against the closed form log1p(sum_j!=y exp(x_j - x_y)) instead)
   aggregation  |g - o| <= 1e-6 * sum_i |w_i x_i[j]|  and  ||g - o||_2 <= 1e-6 ||o||_2

@@ -1,5 +1,5 @@
 """Parity of lsgd_aggregate_round with the CPU oracle: Eq. 3 and its form around x_t, fp32 and bf16 replicas,
-with and without the write-back into the replicas.  Tolerances (fp32 accumulation, derived in the design doc):
+with and without the write-back into the replicas.  Tolerances (fp32 accumulation: one rounding per difference, P fused multiply-adds, one final add):
   plain form   |g - o| <= 1e-6 * sum_i |w_i x_i[j]|
   delta form   |g - o| <= 1e-6 * sum_i |w_i (x_i[j] - b[j])| + 2^-24 * 1.01 * |o|      (the last term: the final add)
   write-back   fp32 replicas hold `out` bit for bit; bf16 replicas hold `out` rounded to nearest even, bit for bit
