@@ -16,12 +16,13 @@
 // Row shapes and their kernels (all bound by the bytes of the logits):
 //   tiny rows   (C <= 32)         one thread per row out of a shared-memory tile
 //   small rows  (<= 2 KB)         4, 8 or 16 lanes per row out of a shared-memory tile
-//   short rows  (<= 4064 bytes)   one warp per row, the row held in registers
-//   long rows   (<= 256 KB)       a ring of 4 KB chunk buffers per SM filled by bulk
+//   medium rows (fp32 <= 256 KB,  one warp per row, streamed through registers with a running (max, sum)
+//                bf16 <= 32 KB)
+//   long rows   (bf16 <= 256 KB)  a ring of 4 KB chunk buffers per SM filled by bulk
 //                                 asynchronous copies (TMA, 1-D); free-running warps
 //                                 reduce chunks to (max, sum) records
 //   anything longer               one CTA per row, two passes over global memory
-// Rows whose label is ignore_index are never scored; the kernels for short, long and longer rows do not even
+// Rows whose label is ignore_index are never scored; the kernels for medium, long and longer rows do not even
 // read them (tiny and small rows are copied tile-wise, ignored rows included).
 #include <cuda_bf16.h>
 
@@ -344,82 +345,164 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
 }
 
 // ---------------------------------------------------------------------------
-// Short rows: one warp per row.  The warp reads the 16-byte-aligned superset of
-// the row (VPL vectors per lane, all loads in flight together), masks what lies
-// outside the row with -inf and keeps the row in registers for both passes.
+// Medium rows (above 2 KB): one warp per row, the row streamed through
+// registers in steps of kStreamU vectors per lane, the next step's loads in
+// flight while the current one is reduced.  Each lane keeps a running maximum
+// m_l and the sum s_l of 2^(x L - p_l), p_l = fl(m_l L), over its elements
+// (L = log2 e); a step that raises the maximum rescales s_l by 2^(p_old - p_new)
+// (the difference of the two rounded products: exact whenever it matters).  At the
+// end  s = 2^-D sum_l s_l 2^(p_l - P),  P = fl(M L), D = M L - P (one fused
+// multiply-add), M = max_l m_l, is sum_j exp(x_j - M).  Rows with s < 1.5
+// (confident ones, where log s would lose the small terms next to the 1 of the
+// maximum) are read once more (cache hits as a rule) and summed with the maximum
+// left out, as in the other kernels.  Whole interior vectors need no masking; the
+// partial vectors in which an unaligned row starts and ends are taken element
+// by element.
 // ---------------------------------------------------------------------------
-constexpr int kWarpThreads = 256;
+constexpr int kStreamThreads = 256;
+constexpr int kStreamU = 4;                       // vectors (16 bytes) per lane and step: 2 KB per warp and step
+constexpr int kStreamMaxRowBytesBf16 = 32 * 1024;
+constexpr int kStreamMaxRowBytesF32 = 256 * 1024;
 
-template <typename T, int VPL>
-__global__ void __launch_bounds__(kWarpThreads)
-score_warp_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
-                       int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0) {
+template <typename T>
+__device__ __forceinline__ void widen_vector(const uint4& q, float (&v)[Elem<T>::kPerVec]) {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+    if constexpr (Elem<T>::kPerVec == 4) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = __uint_as_float(w[e]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            v[2 * e] = __uint_as_float(w[e] << 16);
+            v[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kStreamThreads)
+score_stream_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
+                         int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0) {
     constexpr int EPV = Elem<T>::kPerVec;
+    constexpr int U = kStreamU;
     __shared__ uint32_t hist_s[kSelBins];
     Hist0 h{hist_s, hist0};
     h.clear();
     __syncthreads();
     const int lane = threadIdx.x & 31;
-    const int64_t warps = static_cast<int64_t>(gridDim.x) * (kWarpThreads / 32);
+    const int64_t warps = static_cast<int64_t>(gridDim.x) * (kStreamThreads / 32);
     const int64_t row_bytes = static_cast<int64_t>(C) * sizeof(T);
-    for (int64_t row = static_cast<int64_t>(blockIdx.x) * (kWarpThreads / 32) + (threadIdx.x >> 5); row < rows;
-         row += warps) {
-        const int64_t y = labels[row];
+    const uint4 fill = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);   // -inf in every bf16 slot
+    const uint4 fill32 = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);  // -inf in every fp32 slot
+    const uint4 none = EPV == 4 ? fill32 : fill;
+    int64_t row = static_cast<int64_t>(blockIdx.x) * (kStreamThreads / 32) + (threadIdx.x >> 5);
+    int64_t y = row < rows ? labels[row] : ignore_index;
+    for (; row < rows; row += warps) {
+        const int64_t y_next = row + warps < rows ? labels[row + warps] : ignore_index;  // requested a row ahead
         const int cls = label_class(y, C, ignore_index);
         float loss = 0.f;
         if (cls == 2) {
             loss = __uint_as_float(0x7FC00000u);
             if (lane == 0) atomicAdd(&status->bad_labels, 1);
         } else if (cls == 0) {
-            const uintptr_t ga = reinterpret_cast<uintptr_t>(logits) + row * row_bytes;
+            const T* x_row = logits + row * C;
+            const uintptr_t ga = reinterpret_cast<uintptr_t>(x_row);
             const int head = static_cast<int>(ga & 15);
             const uint4* vbase = reinterpret_cast<const uint4*>(ga - head);
             const int nvec = static_cast<int>((head + row_bytes + 15) >> 4);
-            const int e0 = -head / static_cast<int>(sizeof(T));  // element index of slot 0 of vector 0
-            uint4 raw[VPL];
+            const int tail_bytes = static_cast<int>((head + row_bytes) & 15);  // bytes of the row in its last vector, 0 = all 16
+            const int v_begin = head ? 1 : 0, v_end = tail_bytes ? nvec - 1 : nvec;  // the whole vectors
+            const int n_head = head ? (16 - head) / static_cast<int>(sizeof(T)) : 0;  // elements before them
+            const int n_tail = tail_bytes / static_cast<int>(sizeof(T));              // elements after them
+            const float xy = Elem<T>::widen(__ldg(x_row + y));
+
+            float m = -1e30f, p = -1e30f * kLog2e, s = 0.f;
+            auto fold = [&](const float* v, int n) {  // n new elements (-inf where there is none)
+                float mn = m;
+                for (int e = 0; e < n; ++e) mn = fmaxf(mn, v[e]);
+                const float pn = mn * kLog2e;
+                s *= ex2(p - pn);
+                for (int e = 0; e < n; ++e) s += ex2(fmaf(v[e], kLog2e, -pn));
+                m = mn;
+                p = pn;
+            };
+            uint4 raw[U], nxt[U];
 #pragma unroll
-            for (int u = 0; u < VPL; ++u) {
-                const int v = lane + 32 * u;
-                raw[u] = v < nvec ? __ldcs(vbase + v) : make_uint4(0, 0, 0, 0);
+            for (int u = 0; u < U; ++u) {
+                const int v = v_begin + u * 32 + lane;
+                raw[u] = v < v_end ? __ldcs(vbase + v) : none;
             }
-            const float xy = Elem<T>::widen(__ldg(logits + row * C + y));
-            float x[VPL][EPV];
-            float m = neg_inf();
+            for (int v0 = v_begin; v0 < v_end; v0 += 32 * U) {
 #pragma unroll
-            for (int u = 0; u < VPL; ++u) {
-                const int j0 = e0 + (lane + 32 * u) * EPV;
-                const uint32_t w[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
-#pragma unroll
-                for (int e = 0; e < EPV; ++e) {
-                    float v;
-                    if constexpr (EPV == 4) v = __uint_as_float(w[e]);
-                    else v = __uint_as_float((e & 1) ? (w[e >> 1] & 0xFFFF0000u) : (w[e >> 1] << 16));
-                    const int j = j0 + e;
-                    v = (j >= 0 && j < C) ? v : neg_inf();
-                    x[u][e] = v;
-                    m = fmaxf(m, v);
+                for (int u = 0; u < U; ++u) {  // the next step's vectors
+                    const int v = v0 + 32 * U + u * 32 + lane;
+                    nxt[u] = v < v_end ? __ldcs(vbase + v) : none;
                 }
+                float xv[U * EPV];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    float t[EPV];
+                    widen_vector<T>(raw[u], t);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) xv[u * EPV + e] = t[e];
+                }
+                {
+                    float mn = m;
+#pragma unroll
+                    for (int e = 0; e < U * EPV; ++e) mn = fmaxf(mn, xv[e]);
+                    const float pn = mn * kLog2e;
+                    s *= ex2(p - pn);
+                    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                    for (int e = 0; e < U * EPV; e += 2) {
+                        s0 += ex2(fmaf(xv[e], kLog2e, -pn));
+                        s1 += ex2(fmaf(xv[e + 1], kLog2e, -pn));
+                    }
+                    s += s0 + s1;
+                    m = mn;
+                    p = pn;
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) raw[u] = nxt[u];
             }
-            m = warp_max(m);
-            const RowScale rs(m);
-            float s = 0.f;
-            int n_max = 0;
-#pragma unroll
-            for (int u = 0; u < VPL; ++u)
-#pragma unroll
-                for (int e = 0; e < EPV; ++e) {
-                    const float v = x[u][e];
-                    if (v < m) s += ex2(fmaf(v, kLog2e, rs.nml));
+            if (n_head + n_tail > 0) {  // the partial vectors, one element per lane
+                float v1[1];
+                v1[0] = lane < n_head ? Elem<T>::widen(x_row[lane])
+                        : lane < n_head + n_tail ? Elem<T>::widen(x_row[C - n_tail + (lane - n_head)]) : neg_inf();
+                fold(v1, 1);
+            }
+            const float M = warp_max(m);
+            const float P = M * kLog2e;
+            float sum = warp_sum(s * ex2(p - P));
+            sum *= ex2(-fmaf(M, kLog2e, -P));
+            if (sum >= 1.5f) {
+                loss = (M - xy) + logf(sum);
+            } else {
+                const RowScale rs(M);
+                float s_lt = 0.f;
+                int n_max = 0;
+                auto take = [&](float v) {
+                    if (v < M) s_lt += ex2(fmaf(v, kLog2e, rs.nml));
                     else ++n_max;
+                };
+                for (int v = v_begin + lane; v < v_end; v += 32) {
+                    float t[EPV];
+                    widen_vector<T>(__ldg(vbase + v), t);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) take(t[e]);
                 }
-            s = warp_sum(s);
-            n_max = warp_sum(n_max);
-            loss = finish_loss(m, xy, s, n_max, rs);
+                if (lane < n_head) take(Elem<T>::widen(x_row[lane]));
+                else if (lane < n_head + n_tail) take(Elem<T>::widen(x_row[C - n_tail + (lane - n_head)]));
+                s_lt = warp_sum(s_lt);
+                n_max = warp_sum(n_max);
+                loss = finish_loss(M, xy, s_lt, n_max, rs);
+            }
         }
         if (lane == 0) {
             row_loss[row] = loss;
             h.add(loss);
         }
+        y = y_next;
     }
     __syncthreads();
     h.flush();
@@ -1020,17 +1103,14 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
         return err;
     }
     const int64_t need_vec = (row_bytes + 30) / 16;  // vectors of the aligned superset, worst alignment
-    if (need_vec <= 256) {
-        const int64_t want = (rows + 7) / 8;
-        auto go = [&](auto kernel) {
-            const int grid = static_cast<int>(std::min<int64_t>(want, static_cast<int64_t>(sms) * blocks_per_sm(kernel, kWarpThreads, 0)));
-            kernel<<<grid, kWarpThreads, 0, s>>>(logits, labels, rows, static_cast<int>(C), ignore_index, row_loss,
-                                                 status, hist0);
-        };
-        if (need_vec <= 32) go(score_warp_rows_kernel<T, 1>);
-        else if (need_vec <= 64) go(score_warp_rows_kernel<T, 2>);
-        else if (need_vec <= 128) go(score_warp_rows_kernel<T, 4>);
-        else go(score_warp_rows_kernel<T, 8>);
+    // streamed rows: fp32 up to the ring's limit (measured faster than the ring at every length), bf16 up to 32 KB
+    // (beyond that the ring's two-wide arithmetic wins)
+    if (row_bytes <= (sizeof(T) == 4 ? kStreamMaxRowBytesF32 : kStreamMaxRowBytesBf16)) {
+        const int64_t want = (rows + kStreamThreads / 32 - 1) / (kStreamThreads / 32);
+        const int grid = static_cast<int>(std::min<int64_t>(
+            want, static_cast<int64_t>(sms) * blocks_per_sm(score_stream_rows_kernel<T>, kStreamThreads, 0)));
+        score_stream_rows_kernel<T><<<grid, kStreamThreads, 0, s>>>(logits, labels, rows, static_cast<int>(C),
+                                                                     ignore_index, row_loss, status, hist0);
         return cudaGetLastError();
     }
     if (need_vec <= static_cast<int64_t>(kMaxRecsPerRow) * kChunkVecs) {

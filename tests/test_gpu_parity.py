@@ -59,7 +59,9 @@ SCORE_SHAPES = [
                                                                                  # lane groups: 16/8/4-byte rows or not, 4/8/16 lanes
     (257, 1, 1000, "f32"),
     (65, 3, 1016, "f32"), (40, 2, 2031, "bf16"), (129, 1, 999, "bf16"),          # warp rows, odd alignments
-    (37, 1, 1017, "f32"), (19, 2, 2500, "f32"), (24, 3, 4099, "bf16"), (6, 5, 30522, "bf16"),
+    (37, 1, 1017, "f32"), (19, 2, 2500, "f32"), (24, 3, 4099, "bf16"), (40, 1, 1500, "f32"), (33, 2, 3001, "bf16"),
+    (9, 1, 8191, "f32"), (300, 1, 2048, "bf16"), (21, 1, 16384, "bf16"), (7, 2, 8000, "f32"),  # streamed rows (<= 32 KB)
+    (6, 5, 30522, "bf16"),
     (5, 1, 50001, "f32"),                                                        # CTA rows (shared-memory resident)
     (3, 2, 60011, "f32"), (2, 1, 120013, "bf16"),                                # longer than shared memory
 ]
@@ -97,7 +99,7 @@ def test_score_closed_forms_and_small_losses(L, oracle):
         got = L.score_losses(x, y).cpu().numpy()
         np.testing.assert_allclose(got, np.log(C), rtol=1e-5)
     # confident rows: losses from 1e-1 down to 1e-12 keep their relative accuracy
-    for C in (8, 100, 1000, 6000):
+    for C in (8, 100, 1000, 2500, 6000):
         rows = []
         for gap in (2.0, 5.0, 10.0, 20.0, 30.0):
             r = np.random.default_rng(int(gap)).normal(0, 1, C).astype(np.float32)
