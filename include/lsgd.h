@@ -19,7 +19,7 @@
  *     synchronise, except lsgd_read_device_status.
  *   - Errors are reported by return value only.  Argument errors are found on
  *     the host before anything is launched, so a failing call has no effect on
- *     the device.  No kernel traps or spins without bound.
+ *     the device.  No kernel traps, and no kernel waits on another thread block.
  *   - A size of zero (N == 0, k == 0, D == 0) is legal: the call returns LSGD_OK
  *     without launching anything.
  *   - Workspaces must be 256-byte aligned.  Their contents are scratch: they
@@ -50,7 +50,7 @@ typedef enum lsgd_status {
     LSGD_ERR_ALIGNMENT = 3,   /* pointer not aligned to its element size, workspace not to 256 B      */
     LSGD_ERR_WORKSPACE = 4,   /* ws_bytes smaller than the matching *_workspace_bytes query           */
     LSGD_ERR_CUDA = 5,        /* the CUDA runtime refused a launch or a memset                        */
-    LSGD_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out (reported via the status block)   */
+    LSGD_ERR_TIMEOUT = 6      /* reserved: a bounded device-side wait ran out (no kernel of this version waits) */
 } lsgd_status;
 
 /* Element type of the logits. Labels are always int64, losses always fp32. */
@@ -309,8 +309,8 @@ LSGD_API lsgd_status lsgd_weights_from_steps(const int32_t* tau, int32_t P, floa
  * selection call left at the start of `ws`.  Synchronises `cuda_stream`.
  *   bad_label_count  host, out: tokens whose label was outside [0, C) and not
  *                    ignore_index in that call.
- * Returns LSGD_ERR_TIMEOUT if a bounded device-side wait ran out in that call,
- * LSGD_ERR_CUDA if the copy failed, else LSGD_OK.
+ * Returns LSGD_ERR_CUDA if the copy failed, else LSGD_OK (LSGD_ERR_TIMEOUT is reserved
+ * for kernels with bounded device-side waits; this version has none).
  */
 LSGD_API lsgd_status lsgd_read_device_status(const void* ws, int32_t* bad_label_count, void* cuda_stream);
 

@@ -15,14 +15,15 @@ namespace lsgd {
 // ---------------------------------------------------------------------------
 struct StatusBlock {
     int32_t bad_labels;   // tokens with a label outside [0, C) that is not ignore_index
-    int32_t timeout;      // set when a bounded device-side wait ran out
-    uint32_t row_ticket;  // dynamic row scheduler of the large-row scorer
+    int32_t timeout;      // reserved: set by a kernel whose bounded wait ran out (no kernel of this version waits)
+    uint32_t reserved0;
     // Radix select: CTAs that finished histogram pass p take a ticket; the last one resolves digit p of the
     // threshold key once for everybody: the key prefix with digits 0..p placed, and the rank left inside it.
     uint32_t sel_done[3];
     uint32_t sel_prefix[3];
     uint32_t sel_want[3];
-    uint32_t pad[52];
+    unsigned long long stream_ticket;  // dynamic row scheduler of the medium-row scorer (offset 48)
+    uint32_t pad[50];
 };
 static_assert(sizeof(StatusBlock) == 256, "status block is 256 bytes");
 

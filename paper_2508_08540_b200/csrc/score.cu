@@ -16,13 +16,9 @@
 // Row shapes and their kernels (all bound by the bytes of the logits):
 //   tiny rows   (C <= 32)         one thread per row out of a shared-memory tile
 //   small rows  (<= 2 KB)         4, 8 or 16 lanes per row out of a shared-memory tile
-//   medium rows (fp32 <= 256 KB,  one warp per row, streamed through registers with a running (max, sum)
-//                bf16 <= 32 KB)
-//   long rows   (bf16 <= 256 KB)  a ring of 4 KB chunk buffers per SM filled by bulk
-//                                 asynchronous copies (TMA, 1-D); free-running warps
-//                                 reduce chunks to (max, sum) records
+//   medium rows (<= 256 KB)       one warp per row, streamed through registers with a running (max, sum)
 //   anything longer               one CTA per row, two passes over global memory
-// Rows whose label is ignore_index are never scored; the kernels for medium, long and longer rows do not even
+// Rows whose label is ignore_index are never scored; the kernels for medium and longer rows do not even
 // read them (tiny and small rows are copied tile-wise, ignored rows included).
 #include <cuda_bf16.h>
 
@@ -36,7 +32,6 @@ namespace lsgd {
 namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr uint32_t kWaitLimit = 1u << 20;  // polls (of up to ~2 us each) of a bulk-copy barrier before giving up
 
 __device__ __forceinline__ float ex2(float x) {
     float y;
@@ -345,267 +340,8 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
 }
 
 // ---------------------------------------------------------------------------
-// Medium rows (above 2 KB): one warp per row, the row streamed through
-// registers in steps of kStreamU vectors per lane, the next step's loads in
-// flight while the current one is reduced.  Each lane keeps a running maximum
-// m_l and the sum s_l of 2^(x L - p_l), p_l = fl(m_l L), over its elements
-// (L = log2 e); a step that raises the maximum rescales s_l by 2^(p_old - p_new)
-// (the difference of the two rounded products: exact whenever it matters).  At the
-// end  s = 2^-D sum_l s_l 2^(p_l - P),  P = fl(M L), D = M L - P (one fused
-// multiply-add), M = max_l m_l, is sum_j exp(x_j - M).  Rows with s < 1.5
-// (confident ones, where log s would lose the small terms next to the 1 of the
-// maximum) are read once more (cache hits as a rule) and summed with the maximum
-// left out, as in the other kernels.  Whole interior vectors need no masking; the
-// partial vectors in which an unaligned row starts and ends are taken element
-// by element.
+// Vector arithmetic of the medium-row kernel.
 // ---------------------------------------------------------------------------
-constexpr int kStreamThreads = 256;
-constexpr int kStreamU = 4;                       // vectors (16 bytes) per lane and step: 2 KB per warp and step
-constexpr int kStreamMaxRowBytesBf16 = 32 * 1024;
-constexpr int kStreamMaxRowBytesF32 = 256 * 1024;
-
-template <typename T>
-__device__ __forceinline__ void widen_vector(const uint4& q, float (&v)[Elem<T>::kPerVec]) {
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-    if constexpr (Elem<T>::kPerVec == 4) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) v[e] = __uint_as_float(w[e]);
-    } else {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            v[2 * e] = __uint_as_float(w[e] << 16);
-            v[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
-        }
-    }
-}
-
-template <typename T>
-__global__ void __launch_bounds__(kStreamThreads)
-score_stream_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
-                         int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0) {
-    constexpr int EPV = Elem<T>::kPerVec;
-    constexpr int U = kStreamU;
-    __shared__ uint32_t hist_s[kSelBins];
-    Hist0 h{hist_s, hist0};
-    h.clear();
-    __syncthreads();
-    const int lane = threadIdx.x & 31;
-    const int64_t warps = static_cast<int64_t>(gridDim.x) * (kStreamThreads / 32);
-    const int64_t row_bytes = static_cast<int64_t>(C) * sizeof(T);
-    const uint4 fill = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);   // -inf in every bf16 slot
-    const uint4 fill32 = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);  // -inf in every fp32 slot
-    const uint4 none = EPV == 4 ? fill32 : fill;
-    int64_t row = static_cast<int64_t>(blockIdx.x) * (kStreamThreads / 32) + (threadIdx.x >> 5);
-    int64_t y = row < rows ? labels[row] : ignore_index;
-    for (; row < rows; row += warps) {
-        const int64_t y_next = row + warps < rows ? labels[row + warps] : ignore_index;  // requested a row ahead
-        const int cls = label_class(y, C, ignore_index);
-        float loss = 0.f;
-        if (cls == 2) {
-            loss = __uint_as_float(0x7FC00000u);
-            if (lane == 0) atomicAdd(&status->bad_labels, 1);
-        } else if (cls == 0) {
-            const T* x_row = logits + row * C;
-            const uintptr_t ga = reinterpret_cast<uintptr_t>(x_row);
-            const int head = static_cast<int>(ga & 15);
-            const uint4* vbase = reinterpret_cast<const uint4*>(ga - head);
-            const int nvec = static_cast<int>((head + row_bytes + 15) >> 4);
-            const int tail_bytes = static_cast<int>((head + row_bytes) & 15);  // bytes of the row in its last vector, 0 = all 16
-            const int v_begin = head ? 1 : 0, v_end = tail_bytes ? nvec - 1 : nvec;  // the whole vectors
-            const int n_head = head ? (16 - head) / static_cast<int>(sizeof(T)) : 0;  // elements before them
-            const int n_tail = tail_bytes / static_cast<int>(sizeof(T));              // elements after them
-            const float xy = Elem<T>::widen(__ldg(x_row + y));
-
-            float m = -1e30f, p = -1e30f * kLog2e, s = 0.f;
-            auto fold = [&](const float* v, int n) {  // n new elements (-inf where there is none)
-                float mn = m;
-                for (int e = 0; e < n; ++e) mn = fmaxf(mn, v[e]);
-                const float pn = mn * kLog2e;
-                s *= ex2(p - pn);
-                for (int e = 0; e < n; ++e) s += ex2(fmaf(v[e], kLog2e, -pn));
-                m = mn;
-                p = pn;
-            };
-            uint4 raw[U], nxt[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int v = v_begin + u * 32 + lane;
-                raw[u] = v < v_end ? __ldcs(vbase + v) : none;
-            }
-            for (int v0 = v_begin; v0 < v_end; v0 += 32 * U) {
-#pragma unroll
-                for (int u = 0; u < U; ++u) {  // the next step's vectors
-                    const int v = v0 + 32 * U + u * 32 + lane;
-                    nxt[u] = v < v_end ? __ldcs(vbase + v) : none;
-                }
-                float xv[U * EPV];
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    float t[EPV];
-                    widen_vector<T>(raw[u], t);
-#pragma unroll
-                    for (int e = 0; e < EPV; ++e) xv[u * EPV + e] = t[e];
-                }
-                {
-                    float mn = m;
-#pragma unroll
-                    for (int e = 0; e < U * EPV; ++e) mn = fmaxf(mn, xv[e]);
-                    const float pn = mn * kLog2e;
-                    s *= ex2(p - pn);
-                    float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-                    for (int e = 0; e < U * EPV; e += 2) {
-                        s0 += ex2(fmaf(xv[e], kLog2e, -pn));
-                        s1 += ex2(fmaf(xv[e + 1], kLog2e, -pn));
-                    }
-                    s += s0 + s1;
-                    m = mn;
-                    p = pn;
-                }
-#pragma unroll
-                for (int u = 0; u < U; ++u) raw[u] = nxt[u];
-            }
-            if (n_head + n_tail > 0) {  // the partial vectors, one element per lane
-                float v1[1];
-                v1[0] = lane < n_head ? Elem<T>::widen(x_row[lane])
-                        : lane < n_head + n_tail ? Elem<T>::widen(x_row[C - n_tail + (lane - n_head)]) : neg_inf();
-                fold(v1, 1);
-            }
-            const float M = warp_max(m);
-            const float P = M * kLog2e;
-            float sum = warp_sum(s * ex2(p - P));
-            sum *= ex2(-fmaf(M, kLog2e, -P));
-            if (sum >= 1.5f) {
-                loss = (M - xy) + logf(sum);
-            } else {
-                const RowScale rs(M);
-                float s_lt = 0.f;
-                int n_max = 0;
-                auto take = [&](float v) {
-                    if (v < M) s_lt += ex2(fmaf(v, kLog2e, rs.nml));
-                    else ++n_max;
-                };
-                for (int v = v_begin + lane; v < v_end; v += 32) {
-                    float t[EPV];
-                    widen_vector<T>(__ldg(vbase + v), t);
-#pragma unroll
-                    for (int e = 0; e < EPV; ++e) take(t[e]);
-                }
-                if (lane < n_head) take(Elem<T>::widen(x_row[lane]));
-                else if (lane < n_head + n_tail) take(Elem<T>::widen(x_row[C - n_tail + (lane - n_head)]));
-                s_lt = warp_sum(s_lt);
-                n_max = warp_sum(n_max);
-                loss = finish_loss(M, xy, s_lt, n_max, rs);
-            }
-        }
-        if (lane == 0) {
-            row_loss[row] = loss;
-            h.add(loss);
-        }
-        y = y_next;
-    }
-    __syncthreads();
-    h.flush();
-}
-
-// ---------------------------------------------------------------------------
-// Long rows: a persistent CTA per SM streams rows through a ring of 4 KB chunk
-// buffers in shared memory.
-//   warp 0      producer: takes rows from a device-wide ticket (a batch at a time,
-//               the next batch requested ahead), skips ignored rows, cuts each row
-//               into chunks of 256 vectors and fills the ring with 1-D bulk
-//               asynchronous copies (TMA), tens of chunks ahead of use;
-//   warps 1..   consumers: each takes the next chunk, whichever row it belongs to,
-//               moves it into registers, hands the buffer straight back, and reduces
-//               it to one record (M_c, S_c): the chunk's maximum and its sum of
-//               exp(x - M_c).  Chunks are independent, so warps never wait for each
-//               other and drift apart freely: the special-function unit, which
-//               bounds bf16 rows (one ex2 per 2 bytes), always has warps to serve.
-// The warp that delivers a row's last record combines the records in a fixed
-// order: m = max_c M_c, s = sum_c S_c exp(M_c - m), l = (m - x_y) + log s.
-// If s < 1.5 (a confident row, where log s would lose the small terms next to the 1
-// of the maximum), that warp re-reads the row (an L2 hit as a rule) and sums it with
-// the maximum left out: l = (m - x_y) + log1p(s').
-// Only the vectors that lie wholly inside a row are bulk-copied, so nothing needs
-// masking in the chunk loop; the (at most two) vectors in which a row starts or ends
-// are read element by element by the warp that finishes the row and enter the
-// combination as records of their own.  Nothing outside a row is ever read.
-// No CTA-wide barrier exists; every mbarrier wait is bounded.  Copies complete out
-// of order, so a stage's barrier can be a whole lap behind the chunk a fast warp is
-// asking for: a stage is taken only when its record number is the chunk's.
-// ---------------------------------------------------------------------------
-constexpr int kRingMaxStages = 48;       // 4 KB each
-constexpr int kChunkVecs = 256;          // vectors per chunk: 8 per lane
-constexpr int kChunkBytes = kChunkVecs * 16;
-constexpr int kVecPerLane = kChunkVecs / 32;
-constexpr int kRingBatch = 8;            // rows taken per ticket
-constexpr int kRowSlots = 128;           // rows between their first chunk and their loss (<= stages + warps live at once)
-constexpr int kRecSlots = 256;           // chunk records, by chunk sequence number
-constexpr int kMaxRecsPerRow = 64;       // longer rows (> 256 KB) take the plain kernel
-constexpr int kExpWarps = 24;            // consumer warps
-constexpr int kRingThreads = 32 * (1 + kExpWarps);
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, 2000;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: false if the barrier did not flip within the poll limit.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-// 1-D bulk asynchronous copy global -> shared, completion counted in bytes on `bar`.
-// dst, src 16-byte aligned; bytes a multiple of 16.
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_u32(dst)),
-                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
-}
-
-struct RowSlot {
-    int64_t row;
-    int64_t label;
-    int32_t first_rec;  // sequence number of the row's first chunk record
-    int32_t nrec;       // chunks of the row
-    int32_t count;      // records delivered so far
-    float xy;           // the true-class logit (set by the warp whose chunk holds it)
-};
-struct RingShared {
-    uint64_t full[kRingMaxStages];   // the chunk's bytes have landed (producer + TMA)
-    uint64_t empty[kRingMaxStages];  // the buffer may be refilled (the warp that took the chunk)
-    int32_t c_slot[kRingMaxStages];  // per stage: row slot of the chunk, -1 = stop
-    int32_t c_v0[kRingMaxStages];    // first vector of the chunk within its row
-    int32_t c_nv[kRingMaxStages];    // vectors in the chunk
-    int32_t c_rec[kRingMaxStages];   // record sequence number
-    RowSlot rows[kRowSlots];
-    float rec_max[kRecSlots];
-    float rec_sum[kRecSlots];
-    uint32_t next_chunk;             // chunk sequence number handed to the next free warp
-    int32_t abort;                   // a bounded wait ran out somewhere in this CTA
-};
-constexpr int kRingHeaderBytes = 8192;
-static_assert(sizeof(RingShared) <= kRingHeaderBytes, "ring header");
-
 // Running maximum over vectors: packed bf16 pairs for bf16 rows (exact: a maximum rounds nothing).
 template <typename T>
 struct VecMax;
@@ -684,261 +420,173 @@ __device__ __forceinline__ void vec_sum_exp(const uint4& q, F2 l2e, F2 nml, F2& 
     }
 }
 
+// ---------------------------------------------------------------------------
+// Medium rows (above 2 KB): one warp per row, the row streamed through
+// registers in steps of kStreamU vectors per lane, the next step's loads in
+// flight while the current one is reduced.  Each lane keeps a running maximum
+// m_l and the sum s_l of 2^(x L - p_l), p_l = fl(m_l L), over its elements
+// (L = log2 e); a step that raises the maximum rescales s_l by 2^(p_old - p_new)
+// (the difference of the two rounded products: exact whenever it matters).  At the
+// end  s = 2^-D sum_l s_l 2^(p_l - P),  P = fl(M L), D = M L - P (one fused
+// multiply-add), M = max_l m_l, is sum_j exp(x_j - M).  Rows with s < 1.5
+// (confident ones, where log s would lose the small terms next to the 1 of the
+// maximum) are read once more (cache hits as a rule) and summed with the maximum
+// left out, as in the other kernels.  Whole interior vectors need no masking; the
+// partial vectors in which an unaligned row starts and ends are taken element
+// by element.
+// ---------------------------------------------------------------------------
+constexpr int kStreamThreads = 256;
+constexpr int kStreamU = 4;                       // vectors (16 bytes) per lane and step: 2 KB per warp and step
+constexpr int kStreamMaxRowBytes = 256 * 1024;
+
 template <typename T>
-__global__ void __launch_bounds__(kRingThreads, 1)
-score_ring_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
-                       int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0) {
+__device__ __forceinline__ void widen_vector(const uint4& q, float (&v)[Elem<T>::kPerVec]) {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+    if constexpr (Elem<T>::kPerVec == 4) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = __uint_as_float(w[e]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            v[2 * e] = __uint_as_float(w[e] << 16);
+            v[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kStreamThreads)
+score_stream_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
+                         int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0,
+                         int batch) {
     constexpr int EPV = Elem<T>::kPerVec;
-    constexpr int kStages = kRingMaxStages;
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    RingShared& sh = *reinterpret_cast<RingShared*>(smem_raw);
-    uint32_t* hist_s = reinterpret_cast<uint32_t*>(smem_raw + kRingHeaderBytes);
-    unsigned char* bufs = smem_raw + kRingHeaderBytes + (hist0 ? kSelBins * sizeof(uint32_t) : 0);
+    constexpr int U = kStreamU;
+    __shared__ uint32_t hist_s[kSelBins];
     Hist0 h{hist_s, hist0};
     h.clear();
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t row_bytes = static_cast<int64_t>(C) * sizeof(T);
-    if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(&sh.full[s], 1);
-            mbar_init(&sh.empty[s], 1);
-        }
-        sh.next_chunk = 0;
-        sh.abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
     __syncthreads();
-
-    if (warp == 0) {
-        // ---------------- producer ----------------
-        // The whole warp works in step: lane k pushes chunks k, k + 32, ... of the current row, so a
-        // row's copies are issued side by side; the per-row bookkeeping is lane 0's.
-        uint32_t seq = 0;      // chunk sequence number of the row's first chunk (= its record number)
-        uint32_t row_seq = 0;  // rows pushed so far
-        bool failed = false;
-        // claims the stage of chunk sequence number q; false once a wait has run out
-        auto claim = [&](uint32_t q) -> bool {
-            if (failed || sh.abort) return false;
-            if (!mbar_wait(&sh.empty[q % kStages], ((q / kStages) & 1) ^ 1)) {
-                atomicExch(&status->timeout, 1);
-                sh.abort = 1;
-                failed = true;
-            }
-            return !failed;
-        };
-        auto push_row = [&](int64_t r, int64_t y) {
-            const uintptr_t ga = reinterpret_cast<uintptr_t>(logits) + r * row_bytes;
+    const int lane = threadIdx.x & 31;
+    const int64_t row_bytes = static_cast<int64_t>(C) * sizeof(T);
+    const uint4 fill = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);   // -inf in every bf16 slot
+    const uint4 fill32 = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);  // -inf in every fp32 slot
+    const uint4 none = EPV == 4 ? fill32 : fill;
+    // Rows are handed out in batches from a device-wide ticket (ignored rows cost nothing, so a fixed assignment
+    // would leave warps idle at the end); a warp asks for its next batch before it starts on the current one.
+    auto grab = [&]() -> int64_t {
+        unsigned long long t = 0;
+        if (lane == 0) t = atomicAdd(&status->stream_ticket, static_cast<unsigned long long>(batch));
+        return static_cast<int64_t>(__shfl_sync(0xFFFFFFFFu, t, 0));
+    };
+    int64_t cur = grab(), ahead = grab();
+    int64_t row = cur;
+    int64_t y = row < rows ? labels[row] : ignore_index;
+    while (row < rows) {
+        // the row after this one: the next of the batch, else the first of the batch already granted
+        const bool last_of_batch = row + 1 >= cur + batch || row + 1 >= rows;
+        const int64_t row_next = last_of_batch ? ahead : row + 1;
+        const int64_t y_next = row_next < rows ? labels[row_next] : ignore_index;  // requested a row ahead
+        const int cls = label_class(y, C, ignore_index);
+        float loss = 0.f;
+        if (cls == 2) {
+            loss = __uint_as_float(0x7FC00000u);
+            if (lane == 0) atomicAdd(&status->bad_labels, 1);
+        } else if (cls == 0) {
+            const T* x_row = logits + row * C;
+            const uintptr_t ga = reinterpret_cast<uintptr_t>(x_row);
             const int head = static_cast<int>(ga & 15);
+            const uint4* vbase = reinterpret_cast<const uint4*>(ga - head);
             const int nvec = static_cast<int>((head + row_bytes + 15) >> 4);
-            // only the vectors that lie wholly inside the row travel by bulk copy; the (at most two) vectors in
-            // which the row starts or ends are read element by element by the warp that finishes the row
-            const int first = head ? 1 : 0;
-            const int last = ((head + row_bytes) & 15) ? nvec - 1 : nvec;
-            const int nchunk = (max(last - first, 0) + kChunkVecs - 1) / kChunkVecs;
-            const int slot = row_seq++ % kRowSlots;
-            if (lane == 0) {
-                RowSlot& rs = sh.rows[slot];
-                rs.row = r;
-                rs.label = y;
-                rs.first_rec = static_cast<int32_t>(seq);
-                rs.nrec = nchunk;  // >= 1: rows of this kernel span hundreds of vectors
-                rs.count = 0;
-            }
-            __syncwarp();  // the slot is written before any lane publishes a chunk of the row
-            const unsigned char* src = reinterpret_cast<const unsigned char*>(ga - head);
-            for (int k = lane; k < nchunk; k += 32) {
-                const uint32_t q = seq + k;
-                if (!claim(q)) break;
-                const int s = q % kStages;
-                const int v0 = first + k * kChunkVecs;
-                const int nv = min(kChunkVecs, last - v0);
-                sh.c_slot[s] = slot;
-                sh.c_v0[s] = v0;
-                sh.c_nv[s] = nv;
-                sh.c_rec[s] = static_cast<int32_t>(q);
-                const uint32_t bytes = static_cast<uint32_t>(nv) << 4;
-                mbar_expect_tx(&sh.full[s], bytes);
-                bulk_g2s(bufs + static_cast<size_t>(s) * kChunkBytes, src + (static_cast<size_t>(v0) << 4), bytes,
-                         &sh.full[s]);
-            }
-            seq += nchunk;
-            __syncwarp();
-        };
-        // lane 0 draws the ticket, lanes 0 .. kRingBatch-1 fetch one label each
-        auto take = [&](int64_t& base, int64_t& lab) {
-            uint32_t t = 0;
-            if (lane == 0) t = atomicAdd(&status->row_ticket, static_cast<uint32_t>(kRingBatch));
-            base = static_cast<int64_t>(__shfl_sync(0xFFFFFFFFu, t, 0));
-            lab = (lane < kRingBatch && base + lane < rows) ? labels[base + lane] : ignore_index;
-        };
-        // the ticket and the labels of the NEXT batch are requested before the current batch is
-        // worked through, so their round trips to memory hide behind the copies being issued
-        int64_t next_base, next_lab;
-        take(next_base, next_lab);
-        for (;;) {
-            const int64_t base = next_base, lab = next_lab;
-            if (base >= rows || __any_sync(0xFFFFFFFFu, failed || sh.abort)) break;
-            take(next_base, next_lab);
-            for (int j = 0; j < kRingBatch && base + j < rows; ++j) {
-                const int64_t r = base + j;
-                const int64_t y = __shfl_sync(0xFFFFFFFFu, lab, j);
-                const int cls = label_class(y, C, ignore_index);
-                if (cls == 0) {
-                    push_row(r, y);
-                } else if (lane == 0) {
-                    float l = 0.f;
-                    if (cls == 2) {
-                        l = __uint_as_float(0x7FC00000u);
-                        atomicAdd(&status->bad_labels, 1);
-                    }
-                    row_loss[r] = l;
-                    h.add(l);
-                }
-            }
-        }
-        // stop markers: every consumer warp takes exactly one
-        if (lane < kExpWarps) {
-            const uint32_t q = seq + lane;
-            claim(q);  // after a failed wait nothing is waited for any more
-            sh.c_slot[q % kStages] = -1;
-            sh.c_rec[q % kStages] = static_cast<int32_t>(q);
-            mbar_arrive(&sh.full[q % kStages]);
-        }
-        __syncwarp();
-    } else {
-        // ---------------- consumers ----------------
-        for (;;) {
-            uint32_t c = 0;
-            if (lane == 0) c = atomicAdd(&sh.next_chunk, 1u);
-            c = __shfl_sync(0xFFFFFFFFu, c, 0);
-            const int s = c % kStages;
-            // A parity wait only tells the current phase from the one before it.  Copies complete out of
-            // order, so this warp can get here while the chunk that used the stage one lap earlier
-            // (c - kStages) is still in flight; the barrier is then a whole phase behind and the wait
-            // passes at once.  The stage's record number says which chunk the stage really holds: the
-            // wait is over only when it is this chunk's (the producer writes it before it arrives on the
-            // barrier, and cannot write it before the earlier chunk has been released).
-            bool landed = false;
-            for (uint32_t spin = 0; spin < kWaitLimit; ++spin) {
-                if (!mbar_wait(&sh.full[s], (c / kStages) & 1)) break;  // the bounded wait ran out
-                if (*reinterpret_cast<volatile int32_t*>(&sh.c_rec[s]) == static_cast<int32_t>(c)) {
-                    landed = true;
-                    break;
-                }
-            }
-            if (!landed) {
-                atomicExch(&status->timeout, 1);
-                sh.abort = 1;
-                break;  // no barrier ties this warp to the others: it can simply leave
-            }
-            const int slot = sh.c_slot[s];
-            if (slot < 0) break;
-            RowSlot& rs = sh.rows[slot];
-            const int v0 = sh.c_v0[s], nv = sh.c_nv[s], rec = sh.c_rec[s] % kRecSlots;
-            const int64_t row = rs.row;
-            const uintptr_t ga = reinterpret_cast<uintptr_t>(logits) + row * row_bytes;
-            const int head = static_cast<int>(ga & 15);
-            const int nvec = static_cast<int>((head + row_bytes + 15) >> 4);
-            const int tail = static_cast<int>((head + row_bytes) & 15);  // bytes of the row in its last vector (0 = all 16)
-            const int e0 = -head / static_cast<int>(sizeof(T));          // element index of slot 0 of vector 0
-            const uint4* vec = reinterpret_cast<const uint4*>(bufs + static_cast<size_t>(s) * kChunkBytes);
-            // vector of the true-class logit within the row; it may be one of the two edge vectors
-            const int64_t ey = rs.label - e0;  // element slot counted from the row's first vector
-            const int vy = static_cast<int>(ey / EPV);
+            const int tail_bytes = static_cast<int>((head + row_bytes) & 15);  // bytes of the row in its last vector, 0 = all 16
+            const int v_begin = head ? 1 : 0, v_end = tail_bytes ? nvec - 1 : nvec;  // the whole vectors
+            const int n_head = head ? (16 - head) / static_cast<int>(sizeof(T)) : 0;  // elements before them
+            const int n_tail = tail_bytes / static_cast<int>(sizeof(T));              // elements after them
+            const float xy = Elem<T>::widen(__ldg(x_row + y));
 
-            // -- the chunk into registers: whole vectors of the row only, nothing to mask
-            uint4 raw[kVecPerLane];
-            if (nv == kChunkVecs) {
+            float m = -1e30f, p = -1e30f * kLog2e, s = 0.f;
+            auto fold = [&](const float* v, int n) {  // n new elements (-inf where there is none)
+                float mn = m;
+                for (int e = 0; e < n; ++e) mn = fmaxf(mn, v[e]);
+                const float pn = mn * kLog2e;
+                s *= ex2(p - pn);
+                for (int e = 0; e < n; ++e) s += ex2(fmaf(v[e], kLog2e, -pn));
+                m = mn;
+                p = pn;
+            };
+            uint4 raw[U], nxt[U];
 #pragma unroll
-                for (int u = 0; u < kVecPerLane; ++u) raw[u] = vec[lane + 32 * u];
-            } else {  // the last chunk of a row
-                const uint32_t ninf = EPV == 4 ? 0xFF800000u : 0xFF80FF80u;
+            for (int u = 0; u < U; ++u) {
+                const int v = v_begin + u * 32 + lane;
+                raw[u] = v < v_end ? __ldcs(vbase + v) : none;
+            }
+            for (int v0 = v_begin; v0 < v_end; v0 += 32 * U) {
 #pragma unroll
-                for (int u = 0; u < kVecPerLane; ++u) {
-                    const int i = lane + 32 * u;
-                    raw[u] = i < nv ? vec[i] : make_uint4(ninf, ninf, ninf, ninf);
+                for (int u = 0; u < U; ++u) {  // the next step's vectors
+                    const int v = v0 + 32 * U + u * 32 + lane;
+                    nxt[u] = v < v_end ? __ldcs(vbase + v) : none;
                 }
-            }
-            if (lane == 0 && vy >= v0 && vy < v0 + nv)  // the true-class logit, if this chunk holds it
-                rs.xy = Elem<T>::widen(reinterpret_cast<const T*>(vec)[ey - static_cast<int64_t>(v0) * EPV]);
-
-            // -- chunk maximum (every lane's loads have returned once the shuffles are through)
-            VecMax<T> vm;
+                {
+                    VecMax<T> vm;  // bf16: the maximum is taken on packed pairs, before widening
 #pragma unroll
-            for (int u = 0; u < kVecPerLane; ++u) vm.add(raw[u]);
-            const float M = warp_max(vm.get());
-            if (lane == 0) mbar_arrive(&sh.empty[s]);  // the chunk is in registers: the buffer can be refilled
-
-            // -- chunk sum of exponentials
-            const RowScale sc(M);
-            const F2 l2e = pack2(kLog2e, kLog2e), nml2 = pack2(sc.nml, sc.nml);
-            F2 a0 = pack2(0.f, 0.f), a1 = a0;
+                    for (int u = 0; u < U; ++u) vm.add(raw[u]);
+                    const float mn = fmaxf(m, vm.get());
+                    const float pn = mn * kLog2e;
+                    s *= ex2(p - pn);
+                    const F2 l2e = pack2(kLog2e, kLog2e), nml = pack2(-pn, -pn);
+                    F2 a0 = pack2(0.f, 0.f), a1 = pack2(0.f, 0.f);  // two-wide FMAs and adds
 #pragma unroll
-            for (int u = 0; u < kVecPerLane; ++u) vec_sum_exp<T>(raw[u], l2e, nml2, a0, a1);
-            float p0, p1, p2, p3;
-            unpack2(a0, p0, p1);
-            unpack2(a1, p2, p3);
-            const float S = warp_sum((p0 + p1) + (p2 + p3)) * sc.corr;
-
-            // -- record; the warp that delivers the row's last record finishes the row
-            int last = 0;
-            if (lane == 0) {
-                sh.rec_max[rec] = M;
-                sh.rec_sum[rec] = S;
-                __threadfence_block();
-                last = atomicAdd(&rs.count, 1) == rs.nrec - 1;
-            }
-            last = __shfl_sync(0xFFFFFFFFu, last, 0);
-            if (!last) continue;
-            __threadfence_block();
-            const int nrec = rs.nrec, first = rs.first_rec;
-            const int ia = lane, ib = lane + 32;
-            const float Ma = ia < nrec ? sh.rec_max[(first + ia) % kRecSlots] : neg_inf();
-            const float Mb = ib < nrec ? sh.rec_max[(first + ib) % kRecSlots] : neg_inf();
-            const float Sa = ia < nrec ? sh.rec_sum[(first + ia) % kRecSlots] : 0.f;
-            const float Sb = ib < nrec ? sh.rec_sum[(first + ib) % kRecSlots] : 0.f;
-            // the elements of the (at most two) vectors in which the row starts and ends: lanes 0..7 take the
-            // first vector's slots, lanes 8..15 the last vector's, one element load each
-            float xe = neg_inf();
-            int64_t je = -1;
-            if (lane < 16) {
-                const int slot_e = lane & 7;
-                const bool at_head = lane < 8;
-                if (slot_e < EPV && (at_head ? head != 0 : tail != 0)) {
-                    const int64_t j = e0 + (at_head ? 0 : static_cast<int64_t>(nvec - 1) * EPV) + slot_e;
-                    if (j >= 0 && j < C) {
-                        je = j;
-                        xe = Elem<T>::widen(logits[row * C + j]);
-                    }
+                    for (int u = 0; u < U; ++u) vec_sum_exp<T>(raw[u], l2e, nml, a0, a1);
+                    float t0, t1, t2, t3;
+                    unpack2(a0, t0, t1);
+                    unpack2(a1, t2, t3);
+                    s += (t0 + t1) + (t2 + t3);
+                    m = mn;
+                    p = pn;
                 }
+#pragma unroll
+                for (int u = 0; u < U; ++u) raw[u] = nxt[u];
             }
-            const float m = warp_max(fmaxf(fmaxf(Ma, Mb), xe));
-            const float ssum = warp_sum(Sa * ex2((Ma - m) * kLog2e) + Sb * ex2((Mb - m) * kLog2e) +
-                                        (je >= 0 ? ex2((xe - m) * kLog2e) : 0.f));
-            const bool y_at_edge = (head && vy == 0) || (tail && vy == nvec - 1);
-            const float xy = y_at_edge ? warp_max(je == rs.label ? xe : neg_inf()) : rs.xy;
-            float loss;
-            if (ssum >= 1.5f) {
-                loss = (m - xy) + logf(ssum);
+            if (n_head + n_tail > 0) {  // the partial vectors, one element per lane
+                float v1[1];
+                v1[0] = lane < n_head ? Elem<T>::widen(x_row[lane])
+                        : lane < n_head + n_tail ? Elem<T>::widen(x_row[C - n_tail + (lane - n_head)]) : neg_inf();
+                fold(v1, 1);
+            }
+            const float M = warp_max(m);
+            const float P = M * kLog2e;
+            float sum = warp_sum(s * ex2(p - P));
+            sum *= ex2(-fmaf(M, kLog2e, -P));
+            if (sum >= 1.5f) {
+                loss = (M - xy) + logf(sum);
             } else {
-                // a confident row: the sum again with the maximum left out, from a second read of the row
-                const RowScale fs(m);
-                const T* x = logits + row * C;
+                const RowScale rs(M);
                 float s_lt = 0.f;
                 int n_max = 0;
-                for (int j = lane; j < C; j += 32) {
-                    const float v = Elem<T>::widen(x[j]);
-                    if (v < m) s_lt += ex2(fmaf(v, kLog2e, fs.nml));
+                auto take = [&](float v) {
+                    if (v < M) s_lt += ex2(fmaf(v, kLog2e, rs.nml));
                     else ++n_max;
+                };
+                for (int v = v_begin + lane; v < v_end; v += 32) {
+                    float t[EPV];
+                    widen_vector<T>(__ldg(vbase + v), t);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) take(t[e]);
                 }
+                if (lane < n_head) take(Elem<T>::widen(x_row[lane]));
+                else if (lane < n_head + n_tail) take(Elem<T>::widen(x_row[C - n_tail + (lane - n_head)]));
                 s_lt = warp_sum(s_lt);
                 n_max = warp_sum(n_max);
-                loss = finish_loss(m, xy, s_lt, n_max, fs);
+                loss = finish_loss(M, xy, s_lt, n_max, rs);
             }
-            if (lane == 0) {
-                row_loss[row] = loss;
-                h.add(loss);
-            }
+        }
+        if (lane == 0) {
+            row_loss[row] = loss;
+            h.add(loss);
+        }
+        y = y_next;
+        row = row_next;
+        if (last_of_batch) {
+            cur = ahead;
+            if (cur < rows) ahead = grab();
         }
     }
     __syncthreads();
@@ -946,8 +594,8 @@ score_ring_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
 }
 
 // ---------------------------------------------------------------------------
-// Rows too long for shared memory: one CTA per row, two passes over global
-// memory with plain element loads.  A plain fallback, not a tuned path.
+// Rows beyond 256 KB: one CTA per row, two passes over global memory with plain
+// element loads.  A plain fallback, not a tuned path.
 // ---------------------------------------------------------------------------
 constexpr int kCtaThreads = 256;
 constexpr int kCtaWarps = kCtaThreads / 32;
@@ -1102,29 +750,17 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
         else by_chunk(std::integral_constant<int, 16>{});
         return err;
     }
-    const int64_t need_vec = (row_bytes + 30) / 16;  // vectors of the aligned superset, worst alignment
-    // streamed rows: fp32 up to the ring's limit (measured faster than the ring at every length), bf16 up to 32 KB
-    // (beyond that the ring's two-wide arithmetic wins)
-    if (row_bytes <= (sizeof(T) == 4 ? kStreamMaxRowBytesF32 : kStreamMaxRowBytesBf16)) {
+    if (row_bytes <= kStreamMaxRowBytes) {
         const int64_t want = (rows + kStreamThreads / 32 - 1) / (kStreamThreads / 32);
         const int grid = static_cast<int>(std::min<int64_t>(
             want, static_cast<int64_t>(sms) * blocks_per_sm(score_stream_rows_kernel<T>, kStreamThreads, 0)));
+        // rows per ticket: about 16 KB of logits, so that a ticket's round trip hides behind the batch before it
+        const int batch = static_cast<int>(std::max<int64_t>(1, 16384 / row_bytes));
         score_stream_rows_kernel<T><<<grid, kStreamThreads, 0, s>>>(logits, labels, rows, static_cast<int>(C),
-                                                                     ignore_index, row_loss, status, hist0);
+                                                                     ignore_index, row_loss, status, hist0, batch);
         return cudaGetLastError();
     }
-    if (need_vec <= static_cast<int64_t>(kMaxRecsPerRow) * kChunkVecs) {
-        // ring of chunk buffers in shared memory, one persistent CTA per SM
-        const size_t fixed = kRingHeaderBytes + (hist0 ? kSelBins * sizeof(uint32_t) : 0);
-        const size_t smem = fixed + static_cast<size_t>(kRingMaxStages) * kChunkBytes;
-        const int grid = static_cast<int>(std::min<int64_t>(rows, sms));
-        cudaError_t e = cudaFuncSetAttribute(score_ring_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(kMaxDynSmem));
-        if (e != cudaSuccess) return e;
-        score_ring_rows_kernel<T><<<grid, kRingThreads, smem, s>>>(logits, labels, rows, static_cast<int>(C),
-                                                                   ignore_index, row_loss, status, hist0);
-        return cudaGetLastError();
-    }
+    // longer rows are few per byte: a warp per row would leave most of the machine idle, so a CTA takes each
     const int grid = static_cast<int>(std::min<int64_t>(rows, static_cast<int64_t>(sms) * 8));
     score_huge_rows_kernel<T><<<grid, kCtaThreads, 0, s>>>(logits, labels, rows, C, ignore_index, row_loss, status,
                                                             hist0);

@@ -62,8 +62,9 @@ SCORE_SHAPES = [
     (37, 1, 1017, "f32"), (19, 2, 2500, "f32"), (24, 3, 4099, "bf16"), (40, 1, 1500, "f32"), (33, 2, 3001, "bf16"),
     (9, 1, 8191, "f32"), (300, 1, 2048, "bf16"), (21, 1, 16384, "bf16"), (7, 2, 8000, "f32"),  # streamed rows (<= 32 KB)
     (6, 5, 30522, "bf16"),
-    (5, 1, 50001, "f32"),                                                        # CTA rows (shared-memory resident)
-    (3, 2, 60011, "f32"), (2, 1, 120013, "bf16"),                                # longer than shared memory
+    (5, 1, 50001, "f32"),
+    (3, 2, 60011, "f32"), (2, 1, 120013, "bf16"),                                # the longest streamed rows
+    (2, 1, 70001, "f32"), (3, 1, 140001, "bf16"),                                # beyond 256 KB: one CTA per row
 ]
 
 
