@@ -475,6 +475,54 @@ def launches_per_step(cfg) -> int:
     return n
 
 
+SWEEP_SHAPES = (  # rows, classes, dtype: one row shape per scorer kernel and regime, each pool larger than L2
+    (8_000_000, 48, "f32"), (5_000_000, 100, "f32"), (4_000_000, 200, "f32"), (2_000_000, 500, "f32"),
+    (1_281_167, 1000, "f32"), (640_000, 2000, "f32"), (150_000, 8000, "f32"), (40_000, 30522, "f32"),
+    (6_000_000, 100, "bf16"), (3_000_000, 300, "bf16"), (2_000_000, 1000, "bf16"), (1_000_000, 2000, "bf16"),
+    (400_000, 4000, "bf16"), (300_000, 8000, "bf16"), (100_000, 16000, "bf16"), (131_072, 30522, "bf16"),
+)
+
+
+def run_scorer_sweep(args):
+    """--sweep-scorer: lsgd_score_losses over a range of row lengths (seeded normal logits, sigma 2, uniform labels)."""
+    import torch
+
+    from paper_2508_08540_b200 import lsgd
+
+    torch.cuda.set_device(0)
+    peak, peak_src = measured_peak()
+    out = []
+    for rows, C, dt in SWEEP_SHAPES:
+        tdt = torch.float32 if dt == "f32" else torch.bfloat16
+        g = torch.Generator(device="cuda").manual_seed(MASTER_SWEEP_SEED + C)
+        x = torch.empty((rows, C), dtype=tdt, device="cuda")
+        step = max(1, (1 << 28) // C)
+        for r0 in range(0, rows, step):  # filled in slices: no fp32 copy of the whole pool
+            r1 = min(rows, r0 + step)
+            x[r0:r1] = torch.randn((r1 - r0, C), device="cuda", generator=g).mul_(2.0).to(tdt)
+        y = torch.randint(0, C, (rows,), device="cuda", generator=g)
+        losses = torch.empty(rows, dtype=torch.float32, device="cuda")
+        ws = lsgd.workspace(lsgd.score_workspace_bytes(rows, 1, C), "cuda")
+        for _ in range(3):
+            lsgd.score_losses(x, y, losses=losses, ws=ws)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in ev:
+            a.record()
+            lsgd.score_losses(x, y, losses=losses, ws=ws)
+            b.record()
+        torch.cuda.synchronize()
+        ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
+        nbytes = rows * (C * x.element_size() + 12)
+        out.append({"rows": rows, "C": C, "dtype": dt, "row_bytes": C * x.element_size(), "ms": ms,
+                    "gbs": nbytes / ms / 1e6, "frac_of_measured_hbm": nbytes / ms / 1e6 / peak})
+        del x, y, losses
+    print(json.dumps({"metric": "scorer GB/s by row shape", "unit": "GB/s", "peak": peak, "peak_source": peak_src,
+                      "steps": args.steps, "data": "synthetic", "shapes": out}), flush=True)
+
+
+MASTER_SWEEP_SEED = 20250808
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -483,6 +531,8 @@ def main():
     ap.add_argument("--config", type=int, default=4, choices=sorted(wl.CONFIGS))
     ap.add_argument("--impl", default="lsgd", choices=["lsgd", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep-scorer", action="store_true",
+                    help="instead of the round: time lsgd_score_losses alone over a range of row lengths (1 GPU)")
     ap.add_argument("--no-round", action="store_true", help="skip the lsgd_aggregate_round legs (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--n-samples", type=int, default=0, help="profiling: shrink the pool to this many samples")
@@ -492,7 +542,10 @@ def main():
     if args.n_samples or args.d_params:
         n = args.n_samples or cfg.N
         cfg = wl.scaled(cfg, name=cfg.name + "-scaled", N=n, k=max(1, cfg.k * n // cfg.N), D=args.d_params or cfg.D)
-    if args.impl == "reference":
+    if args.sweep_scorer:
+        args.steps = min(args.steps, 20)
+        run_scorer_sweep(args)
+    elif args.impl == "reference":
         run_reference(args, cfg)
     else:
         run_gpu(args, cfg)

@@ -754,8 +754,8 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
         const int64_t want = (rows + kStreamThreads / 32 - 1) / (kStreamThreads / 32);
         const int grid = static_cast<int>(std::min<int64_t>(
             want, static_cast<int64_t>(sms) * blocks_per_sm(score_stream_rows_kernel<T>, kStreamThreads, 0)));
-        // rows per ticket: about 16 KB of logits, so that a ticket's round trip hides behind the batch before it
-        const int batch = static_cast<int>(std::max<int64_t>(1, 16384 / row_bytes));
+        // rows per ticket: about 32 KB of logits
+        const int batch = static_cast<int>(std::max<int64_t>(1, 32768 / row_bytes));
         score_stream_rows_kernel<T><<<grid, kStreamThreads, 0, s>>>(logits, labels, rows, static_cast<int>(C),
                                                                      ignore_index, row_loss, status, hist0, batch);
         return cudaGetLastError();
