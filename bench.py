@@ -484,7 +484,8 @@ SWEEP_SHAPES = (  # rows, classes, dtype: one row shape per scorer kernel and re
 
 
 def run_scorer_sweep(args):
-    """--sweep-scorer: lsgd_score_losses over a range of row lengths (seeded normal logits, sigma 2, uniform labels)."""
+    """--sweep-scorer: lsgd_score_losses over a range of row lengths (seeded normal logits, sigma 2, uniform labels),
+    and some of them again with confident rows."""
     import torch
 
     from paper_2508_08540_b200 import lsgd
@@ -492,15 +493,24 @@ def run_scorer_sweep(args):
     torch.cuda.set_device(0)
     peak, peak_src = measured_peak()
     out = []
-    for rows, C, dt in SWEEP_SHAPES:
+    shapes = [(r, C, dt, 0.0) for r, C, dt in SWEEP_SHAPES]
+    # the same pools from a model that is sure of its answer (true class + 14: p > 0.99, losses ~ 1e-3): the regime
+    # in which the loss keeps its relative accuracy only through the max-excluded sum
+    shapes += [(r, C, dt, 14.0) for r, C, dt in SWEEP_SHAPES if (C, dt) in ((100, "f32"), (1000, "f32"), (8000, "f32"),
+                                                                           (300, "bf16"), (4000, "bf16"), (30522, "bf16"))]
+    for rows, C, dt, bump in shapes:
         tdt = torch.float32 if dt == "f32" else torch.bfloat16
         g = torch.Generator(device="cuda").manual_seed(MASTER_SWEEP_SEED + C)
         x = torch.empty((rows, C), dtype=tdt, device="cuda")
+        y = torch.randint(0, C, (rows,), device="cuda", generator=g)
         step = max(1, (1 << 28) // C)
         for r0 in range(0, rows, step):  # filled in slices: no fp32 copy of the whole pool
             r1 = min(rows, r0 + step)
-            x[r0:r1] = torch.randn((r1 - r0, C), device="cuda", generator=g).mul_(2.0).to(tdt)
-        y = torch.randint(0, C, (rows,), device="cuda", generator=g)
+            blk = torch.randn((r1 - r0, C), device="cuda", generator=g).mul_(2.0)
+            if bump:
+                blk[torch.arange(r1 - r0, device="cuda"), y[r0:r1]] += bump
+            x[r0:r1] = blk.to(tdt)
+            del blk
         losses = torch.empty(rows, dtype=torch.float32, device="cuda")
         ws = lsgd.workspace(lsgd.score_workspace_bytes(rows, 1, C), "cuda")
         for _ in range(3):
@@ -513,7 +523,7 @@ def run_scorer_sweep(args):
         torch.cuda.synchronize()
         ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
         nbytes = rows * (C * x.element_size() + 12)
-        out.append({"rows": rows, "C": C, "dtype": dt, "row_bytes": C * x.element_size(), "ms": ms,
+        out.append({"rows": rows, "C": C, "dtype": dt, "true_class_bump": bump, "row_bytes": C * x.element_size(), "ms": ms,
                     "gbs": nbytes / ms / 1e6, "frac_of_measured_hbm": nbytes / ms / 1e6 / peak})
         del x, y, losses
     print(json.dumps({"metric": "scorer GB/s by row shape", "unit": "GB/s", "peak": peak, "peak_source": peak_src,

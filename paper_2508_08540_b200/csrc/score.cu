@@ -420,20 +420,43 @@ __device__ __forceinline__ void vec_sum_exp(const uint4& q, F2 l2e, F2 nml, F2& 
     }
 }
 
+// Sets slot e of a vector to -inf.
+template <typename T>
+__device__ __forceinline__ uint32_t blank_word(uint32_t w, int i, int e) {
+    if constexpr (sizeof(T) == 4) return i == e ? 0xFF800000u : w;
+    else return i != (e >> 1) ? w : (e & 1) ? ((w & 0x0000FFFFu) | 0xFF800000u) : ((w & 0xFFFF0000u) | 0x0000FF80u);
+}
+template <typename T>
+__device__ __forceinline__ void blank_slot(uint4& q, int e) {
+    q.x = blank_word<T>(q.x, 0, e);
+    q.y = blank_word<T>(q.y, 1, e);
+    q.z = blank_word<T>(q.z, 2, e);
+    q.w = blank_word<T>(q.w, 3, e);
+}
+
+// The loss from the sum over the OTHER classes.  With M = max_{j != y} x_j, P = fl(M L) and
+// S = sum_{j != y} 2^(x_j L - P) (= 2^D sum_{j != y} exp(x_j - M), D = M L - P; S = 0 if there is no other class):
+//   x_y >= M:  l = log1p(sum_{j != y} exp(x_j - x_y)) = log1p(S 2^(P - x_y L))            (one fused multiply-add)
+//   x_y <  M:  l = (M - x_y) + log(sum_j exp(x_j - M)) = (M - x_y) + log((S + 2^(x_y L - P)) 2^-D)
+// Only sums of positive terms: nothing cancels, so a loss of 1e-9 is as accurate as a loss of 10, in one pass and
+// without a comparison per element (a small loss means that the true class dominates, so it is the true class, not
+// the maximum, that has to stay out of the sum).
+__device__ __forceinline__ float loss_without_true_class(float M, float P, float S, float xy) {
+    if (xy >= M) return log1pf(S * ex2(fmaf(-xy, kLog2e, P)));
+    const float D = fmaf(M, kLog2e, -P);
+    return (M - xy) + logf((S + ex2(fmaf(xy, kLog2e, -P))) * ex2(-D));
+}
+
 // ---------------------------------------------------------------------------
 // Medium rows (above 2 KB): one warp per row, the row streamed through
 // registers in steps of kStreamU vectors per lane, the next step's loads in
 // flight while the current one is reduced.  Each lane keeps a running maximum
 // m_l and the sum s_l of 2^(x L - p_l), p_l = fl(m_l L), over its elements
-// (L = log2 e); a step that raises the maximum rescales s_l by 2^(p_old - p_new)
-// (the difference of the two rounded products: exact whenever it matters).  At the
-// end  s = 2^-D sum_l s_l 2^(p_l - P),  P = fl(M L), D = M L - P (one fused
-// multiply-add), M = max_l m_l, is sum_j exp(x_j - M).  Rows with s < 1.5
-// (confident ones, where log s would lose the small terms next to the 1 of the
-// maximum) are read once more (cache hits as a rule) and summed with the maximum
-// left out, as in the other kernels.  Whole interior vectors need no masking; the
-// partial vectors in which an unaligned row starts and ends are taken element
-// by element.
+// (L = log2 e; the true class is left out); a step that raises the maximum
+// rescales s_l by 2^(p_old - p_new) (the difference of the two rounded products:
+// exact whenever it matters).  At the end  S = sum_l s_l 2^(p_l - P),  P = fl(M L),
+// M = max_l m_l.  Whole interior vectors need no masking; the partial vectors in
+// which an unaligned row starts and ends are taken element by element.
 // ---------------------------------------------------------------------------
 constexpr int kStreamThreads = 256;
 constexpr int kStreamU = 4;                       // vectors (16 bytes) per lane and step: 2 KB per warp and step
@@ -502,16 +525,13 @@ score_stream_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict
             const int n_tail = tail_bytes / static_cast<int>(sizeof(T));              // elements after them
             const float xy = Elem<T>::widen(__ldg(x_row + y));
 
+            // The true class is left out of the sum (its slot is blanked to -inf as its vector passes by), which is
+            // all that the relative accuracy of tiny losses needs: see loss_without_true_class.
+            const int y_byte = head + static_cast<int>(y) * static_cast<int>(sizeof(T));
+            const int vy = y_byte >> 4;                                           // the vector that holds x_y ...
+            const int ey = (y_byte & 15) / static_cast<int>(sizeof(T));           // ... and its slot there
+            // Lane state: m (maximum so far), p = fl(m L), s = sum of 2^(x L - p) over the lane's elements so far.
             float m = -1e30f, p = -1e30f * kLog2e, s = 0.f;
-            auto fold = [&](const float* v, int n) {  // n new elements (-inf where there is none)
-                float mn = m;
-                for (int e = 0; e < n; ++e) mn = fmaxf(mn, v[e]);
-                const float pn = mn * kLog2e;
-                s *= ex2(p - pn);
-                for (int e = 0; e < n; ++e) s += ex2(fmaf(v[e], kLog2e, -pn));
-                m = mn;
-                p = pn;
-            };
             uint4 raw[U], nxt[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
@@ -524,13 +544,16 @@ score_stream_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict
                     const int v = v0 + 32 * U + u * 32 + lane;
                     nxt[u] = v < v_end ? __ldcs(vbase + v) : none;
                 }
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (v0 + u * 32 + lane == vy) blank_slot<T>(raw[u], ey);
                 {
                     VecMax<T> vm;  // bf16: the maximum is taken on packed pairs, before widening
 #pragma unroll
                     for (int u = 0; u < U; ++u) vm.add(raw[u]);
                     const float mn = fmaxf(m, vm.get());
                     const float pn = mn * kLog2e;
-                    s *= ex2(p - pn);
+                    s *= ex2(p - pn);  // the maximum rose: rescale (exactly 1 otherwise)
                     const F2 l2e = pack2(kLog2e, kLog2e), nml = pack2(-pn, -pn);
                     F2 a0 = pack2(0.f, 0.f), a1 = pack2(0.f, 0.f);  // two-wide FMAs and adds
 #pragma unroll
@@ -546,37 +569,17 @@ score_stream_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict
                 for (int u = 0; u < U; ++u) raw[u] = nxt[u];
             }
             if (n_head + n_tail > 0) {  // the partial vectors, one element per lane
-                float v1[1];
-                v1[0] = lane < n_head ? Elem<T>::widen(x_row[lane])
-                        : lane < n_head + n_tail ? Elem<T>::widen(x_row[C - n_tail + (lane - n_head)]) : neg_inf();
-                fold(v1, 1);
+                const int j = lane < n_head ? lane : lane < n_head + n_tail ? C - n_tail + (lane - n_head) : -1;
+                const float v = (j >= 0 && j != static_cast<int>(y)) ? Elem<T>::widen(x_row[j]) : neg_inf();
+                const float mn = fmaxf(m, v);
+                const float pn = mn * kLog2e;
+                s = s * ex2(p - pn) + ex2(fmaf(v, kLog2e, -pn));
+                m = mn;
+                p = pn;
             }
             const float M = warp_max(m);
             const float P = M * kLog2e;
-            float sum = warp_sum(s * ex2(p - P));
-            sum *= ex2(-fmaf(M, kLog2e, -P));
-            if (sum >= 1.5f) {
-                loss = (M - xy) + logf(sum);
-            } else {
-                const RowScale rs(M);
-                float s_lt = 0.f;
-                int n_max = 0;
-                auto take = [&](float v) {
-                    if (v < M) s_lt += ex2(fmaf(v, kLog2e, rs.nml));
-                    else ++n_max;
-                };
-                for (int v = v_begin + lane; v < v_end; v += 32) {
-                    float t[EPV];
-                    widen_vector<T>(__ldg(vbase + v), t);
-#pragma unroll
-                    for (int e = 0; e < EPV; ++e) take(t[e]);
-                }
-                if (lane < n_head) take(Elem<T>::widen(x_row[lane]));
-                else if (lane < n_head + n_tail) take(Elem<T>::widen(x_row[C - n_tail + (lane - n_head)]));
-                s_lt = warp_sum(s_lt);
-                n_max = warp_sum(n_max);
-                loss = finish_loss(M, xy, s_lt, n_max, rs);
-            }
+            loss = loss_without_true_class(M, P, warp_sum(s * ex2(p - P)), xy);
         }
         if (lane == 0) {
             row_loss[row] = loss;
