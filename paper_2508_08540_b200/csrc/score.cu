@@ -98,249 +98,8 @@ __device__ __forceinline__ int label_class(int64_t y, int64_t C, int64_t ignore_
 }
 
 // ---------------------------------------------------------------------------
-// Tiny rows: a CTA stages 256 consecutive rows (contiguous in memory) into
-// shared memory with coalesced element loads; each thread then owns one row.
-// ---------------------------------------------------------------------------
-constexpr int kTinyThreads = 256;
-constexpr int kTinyMaxC = 32;
-
-template <typename T>
-__global__ void __launch_bounds__(kTinyThreads)
-score_tiny_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
-                       int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0) {
-    __shared__ float tile[kTinyThreads * (kTinyMaxC + 1)];
-    __shared__ uint32_t hist_s[kSelBins];
-    Hist0 h{hist_s, hist0};
-    h.clear();
-    const int pitch = C | 1;  // odd pitch: conflict-free row reads
-    const int64_t tiles = (rows + kTinyThreads - 1) / kTinyThreads;
-    for (int64_t t = blockIdx.x; t < tiles; t += gridDim.x) {
-        const int64_t row0 = t * kTinyThreads;
-        const int nrows = rows - row0 < kTinyThreads ? static_cast<int>(rows - row0) : kTinyThreads;
-        const T* src = logits + row0 * C;
-        const int n = nrows * C;
-        __syncthreads();
-        for (int i = threadIdx.x; i < n; i += kTinyThreads) {
-            const int r = i / C;
-            tile[r * pitch + (i - r * C)] = Elem<T>::widen(src[i]);
-        }
-        __syncthreads();
-        if (threadIdx.x < nrows) {
-            const int64_t row = row0 + threadIdx.x;
-            const int64_t y = labels[row];
-            const int cls = label_class(y, C, ignore_index);
-            float loss = 0.f;
-            if (cls == 2) {
-                loss = __uint_as_float(0x7FC00000u);
-                atomicAdd(&status->bad_labels, 1);
-            } else if (cls == 0) {
-                const float* x = tile + threadIdx.x * pitch;
-                float m = x[0];
-                for (int j = 1; j < C; ++j) m = fmaxf(m, x[j]);
-                const RowScale rs(m);
-                float s = 0.f;
-                int n_max = 0;
-                for (int j = 0; j < C; ++j) {
-                    const float v = x[j];
-                    if (v < m) s += ex2(fmaf(v, kLog2e, rs.nml));
-                    else ++n_max;
-                }
-                loss = finish_loss(m, x[static_cast<int>(y)], s, n_max, rs);
-            }
-            row_loss[row] = loss;
-            h.add(loss);
-        }
-    }
-    __syncthreads();
-    h.flush();
-}
-
-// ---------------------------------------------------------------------------
-// Small rows (C > 32, at most 2 KB): a CTA copies a tile of consecutive rows (one
-// contiguous, 16-byte-aligned-superset byte range) into shared memory with
-// vector loads; groups of L lanes then own one row each and read it from there.
-// One warp per row would spend most of its instructions on 32-lane reductions
-// and on the per-row epilogue; with L lanes per row those are shared by 32 / L
-// rows.  With a 16-byte-aligned base, rows start on 16-, 8- or 4-byte boundaries
-// according to their length, and a lane reads chunks of that size, l, l + L, ...
-// of its row; otherwise it reads elements l, l + L, ...
-// ---------------------------------------------------------------------------
-constexpr int kGroupThreads = 256;
-constexpr int kGroupMaxRowBytes = 2048;
-constexpr int kGroupStages = 2;
-
-// A chunk: the CB bytes (16, 8 or 4) a lane reads from shared memory at once, CB / sizeof(T) elements.
-template <int CB>
-struct ChunkWord;
-template <>
-struct ChunkWord<16> { using type = uint4; };
-template <>
-struct ChunkWord<8> { using type = uint2; };
-template <>
-struct ChunkWord<4> { using type = uint32_t; };
-
-template <typename T, int CB>
-__device__ __forceinline__ void unpack_chunk(const typename ChunkWord<CB>::type& q, float (&v)[CB / static_cast<int>(sizeof(T))]) {
-    uint32_t w[CB / 4];
-    if constexpr (CB == 16) { w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w; }
-    else if constexpr (CB == 8) { w[0] = q.x; w[1] = q.y; }
-    else { w[0] = q; }
-    if constexpr (sizeof(T) == 4) {
-#pragma unroll
-        for (int e = 0; e < CB / 4; ++e) v[e] = __uint_as_float(w[e]);
-    } else {
-#pragma unroll
-        for (int e = 0; e < CB / 4; ++e) {  // bf16 is the upper half of an fp32
-            v[2 * e] = __uint_as_float(w[e] << 16);
-            v[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
-        }
-    }
-}
-
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst))),
-                 "l"(gsrc)
-                 : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int PENDING>
-__device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
-}
-
-// Tiles flow through a ring of kGroupStages buffers filled by asynchronous 16-byte copies (global -> shared, past
-// the registers), one tile ahead of the one being reduced, so every CTA always has loads in flight; two stages
-// rather than three leave room for a third CTA per SM, which is worth more (measured).
-template <typename T, int L, int CB>
-__global__ void __launch_bounds__(kGroupThreads)
-score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
-                        int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0,
-                        int stage_bytes) {
-    constexpr int R = kGroupThreads / L;  // rows per tile = lane groups per CTA
-    constexpr bool VEC = CB > 0;          // rows start on CB-byte boundaries and are whole chunks (base 16-byte aligned)
-    constexpr bool PADDED = CB == 16 && L < 8;
-    constexpr int EPV = VEC ? CB / static_cast<int>(sizeof(T)) : 1;
-    extern __shared__ __align__(16) unsigned char group_smem[];
-    uint32_t* hist_s = reinterpret_cast<uint32_t*>(group_smem);
-    unsigned char* stages = group_smem + kSelBins * sizeof(uint32_t);
-    Hist0 h{hist_s, hist0};
-    h.clear();
-    const int row_bytes = C * static_cast<int>(sizeof(T));
-    const int64_t tiles = (rows + R - 1) / R;
-    const int g = threadIdx.x / L, l = threadIdx.x % L;
-    // 16-byte chunks, L == 4: two rows share a quarter-warp's accesses, so rows are laid out in shared memory with
-    // a pitch of 4 (mod 8) chunks, which puts neighbouring rows four bank groups apart whatever the row length.
-    // (The order in which a row's elements are summed must not depend on where the row sits: copies of a row
-    // have to score the same bits.)
-    const int nchunk = VEC ? row_bytes / (VEC ? CB : 1) : 0;
-    const int pitch_bytes = PADDED ? 16 * (nchunk + ((L - nchunk) & 7)) : row_bytes;
-    const float inv_nchunk = 1.0f / static_cast<float>(nchunk > 0 ? nchunk : 1);
-    const int64_t my_tiles = tiles > blockIdx.x ? (tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-
-    auto issue = [&](int64_t i) {  // requests this CTA's i-th tile into stage i % kGroupStages
-        if (i < my_tiles) {
-            const int64_t row0 = (blockIdx.x + i * gridDim.x) * R;
-            const int nrows = rows - row0 < R ? static_cast<int>(rows - row0) : R;
-            const uintptr_t b0 = reinterpret_cast<uintptr_t>(logits) + row0 * row_bytes;
-            const int head = VEC ? 0 : static_cast<int>(b0 & 15);
-            const uint4* src = reinterpret_cast<const uint4*>(b0 - head);
-            const int nvec = (head + nrows * row_bytes + 15) >> 4;  // an aligned block that holds a valid byte is safe to read
-            uint4* dst = reinterpret_cast<uint4*>(stages + (i % kGroupStages) * stage_bytes);
-            for (int v = threadIdx.x; v < nvec; v += kGroupThreads) {
-                int d = v;
-                if constexpr (PADDED) {
-                    const int r = __float2int_rz((static_cast<float>(v) + 0.5f) * inv_nchunk);  // v / nchunk, exact here
-                    d = r * (pitch_bytes >> 4) + (v - r * nchunk);
-                }
-                cp_async16(dst + d, src + v);
-            }
-        }
-        cp_async_commit();  // one group per tile slot, also when it is empty: the wait below counts groups
-    };
-    auto label_of = [&](int64_t i) -> int64_t {
-        if (i >= my_tiles) return ignore_index;
-        const int64_t row = (blockIdx.x + i * gridDim.x) * R + g;
-        return row < rows ? labels[row] : ignore_index;
-    };
-
-#pragma unroll
-    for (int i = 0; i < kGroupStages - 1; ++i) issue(i);
-    int64_t y = label_of(0);
-    for (int64_t i = 0; i < my_tiles; ++i) {
-        issue(i + kGroupStages - 1);
-        const int64_t y_next = label_of(i + 1);
-        cp_async_wait<kGroupStages - 1>();
-        __syncthreads();  // everybody's copies of tile i have landed
-        const int64_t row0 = (blockIdx.x + i * gridDim.x) * R;
-        const bool mine = row0 + g < rows;
-        const int head = VEC ? 0 : static_cast<int>((reinterpret_cast<uintptr_t>(logits) + row0 * row_bytes) & 15);
-        const unsigned char* buf = stages + (i % kGroupStages) * stage_bytes;
-        const int cls = mine ? label_class(y, C, ignore_index) : 1;
-        const T* x = reinterpret_cast<const T*>(buf + head + g * pitch_bytes);
-        float m = neg_inf(), s = 0.f;
-        int n_max = 0;
-        if constexpr (VEC) {
-            using Word = typename ChunkWord<VEC ? CB : 16>::type;
-            const Word* xv = reinterpret_cast<const Word*>(x);
-            const int nch = cls == 0 ? nchunk : 0;  // groups without a row to score run the reductions on nothing
-#pragma unroll 2
-            for (int c = l; c < nch; c += L) {
-                float v[EPV];
-                unpack_chunk<T, VEC ? CB : 16>(xv[c], v);
-#pragma unroll
-                for (int e = 0; e < EPV; ++e) m = fmaxf(m, v[e]);
-            }
-#pragma unroll
-            for (int o = L / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-            const RowScale rs(m);
-#pragma unroll 2
-            for (int c = l; c < nch; c += L) {
-                float v[EPV];
-                unpack_chunk<T, VEC ? CB : 16>(xv[c], v);
-#pragma unroll
-                for (int e = 0; e < EPV; ++e) {
-                    if (v[e] < m) s += ex2(fmaf(v[e], kLog2e, rs.nml));
-                    else ++n_max;
-                }
-            }
-        } else {
-            const int n = cls == 0 ? C : 0;
-            for (int j = l; j < n; j += L) m = fmaxf(m, Elem<T>::widen(x[j]));
-#pragma unroll
-            for (int o = L / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-            const RowScale rs(m);
-            for (int j = l; j < n; j += L) {
-                const float v = Elem<T>::widen(x[j]);
-                if (v < m) s += ex2(fmaf(v, kLog2e, rs.nml));
-                else ++n_max;
-            }
-        }
-#pragma unroll
-        for (int o = L / 2; o > 0; o >>= 1) {
-            s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
-            n_max += __shfl_xor_sync(0xFFFFFFFFu, n_max, o);
-        }
-        if (mine && l == 0) {
-            float loss = 0.f;
-            if (cls == 2) {
-                loss = __uint_as_float(0x7FC00000u);
-                atomicAdd(&status->bad_labels, 1);
-            } else if (cls == 0) {
-                loss = finish_loss(m, Elem<T>::widen(x[static_cast<int>(y)]), s, n_max, RowScale(m));
-            }
-            row_loss[row0 + g] = loss;
-            h.add(loss);
-        }
-        __syncthreads();  // the stage may be refilled
-        y = y_next;
-    }
-    cp_async_wait<0>();
-    __syncthreads();
-    h.flush();
-}
-
-// ---------------------------------------------------------------------------
-// Vector arithmetic of the medium-row kernel.
+// Vector arithmetic shared by the kernels for small and medium rows, and the loss
+// formula they end in.
 // ---------------------------------------------------------------------------
 // Running maximum over vectors: packed bf16 pairs for bf16 rows (exact: a maximum rounds nothing).
 template <typename T>
@@ -445,6 +204,273 @@ __device__ __forceinline__ float loss_without_true_class(float M, float P, float
     if (xy >= M) return log1pf(S * ex2(fmaf(-xy, kLog2e, P)));
     const float D = fmaf(M, kLog2e, -P);
     return (M - xy) + logf((S + ex2(fmaf(xy, kLog2e, -P))) * ex2(-D));
+}
+
+// ---------------------------------------------------------------------------
+// Tiny rows: a CTA stages 256 consecutive rows (contiguous in memory) into
+// shared memory with coalesced element loads; each thread then owns one row.
+// ---------------------------------------------------------------------------
+constexpr int kTinyThreads = 256;
+constexpr int kTinyMaxC = 32;
+
+template <typename T>
+__global__ void __launch_bounds__(kTinyThreads)
+score_tiny_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
+                       int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0) {
+    __shared__ float tile[kTinyThreads * (kTinyMaxC + 1)];
+    __shared__ uint32_t hist_s[kSelBins];
+    Hist0 h{hist_s, hist0};
+    h.clear();
+    const int pitch = C | 1;  // odd pitch: conflict-free row reads
+    const int64_t tiles = (rows + kTinyThreads - 1) / kTinyThreads;
+    for (int64_t t = blockIdx.x; t < tiles; t += gridDim.x) {
+        const int64_t row0 = t * kTinyThreads;
+        const int nrows = rows - row0 < kTinyThreads ? static_cast<int>(rows - row0) : kTinyThreads;
+        const T* src = logits + row0 * C;
+        const int n = nrows * C;
+        __syncthreads();
+        for (int i = threadIdx.x; i < n; i += kTinyThreads) {
+            const int r = i / C;
+            tile[r * pitch + (i - r * C)] = Elem<T>::widen(src[i]);
+        }
+        __syncthreads();
+        if (threadIdx.x < nrows) {
+            const int64_t row = row0 + threadIdx.x;
+            const int64_t y = labels[row];
+            const int cls = label_class(y, C, ignore_index);
+            float loss = 0.f;
+            if (cls == 2) {
+                loss = __uint_as_float(0x7FC00000u);
+                atomicAdd(&status->bad_labels, 1);
+            } else if (cls == 0) {
+                const float* x = tile + threadIdx.x * pitch;
+                float m = x[0];
+                for (int j = 1; j < C; ++j) m = fmaxf(m, x[j]);
+                const RowScale rs(m);
+                float s = 0.f;
+                int n_max = 0;
+                for (int j = 0; j < C; ++j) {
+                    const float v = x[j];
+                    if (v < m) s += ex2(fmaf(v, kLog2e, rs.nml));
+                    else ++n_max;
+                }
+                loss = finish_loss(m, x[static_cast<int>(y)], s, n_max, rs);
+            }
+            row_loss[row] = loss;
+            h.add(loss);
+        }
+    }
+    __syncthreads();
+    h.flush();
+}
+
+// ---------------------------------------------------------------------------
+// Small rows (C > 32, at most 2 KB): a CTA copies a tile of consecutive rows (one
+// contiguous, 16-byte-aligned-superset byte range) into shared memory with
+// vector loads; groups of L lanes then own one row each and read it from there.
+// One warp per row would spend most of its instructions on 32-lane reductions
+// and on the per-row epilogue; with L lanes per row those are shared by 32 / L
+// rows.  With a 16-byte-aligned base, rows start on 16-, 8- or 4-byte boundaries
+// according to their length, and a lane reads chunks of that size, l, l + L, ...
+// of its row; otherwise it reads elements l, l + L, ...
+// ---------------------------------------------------------------------------
+constexpr int kGroupThreads = 256;
+constexpr int kGroupMaxRowBytes = 2048;
+constexpr int kGroupStages = 2;
+
+// A chunk: the CB bytes (16, 8 or 4) a lane reads from shared memory at once, CB / sizeof(T) elements.
+template <int CB>
+struct ChunkWord;
+template <>
+struct ChunkWord<16> { using type = uint4; };
+template <>
+struct ChunkWord<8> { using type = uint2; };
+template <>
+struct ChunkWord<4> { using type = uint32_t; };
+
+template <typename T, int CB>
+__device__ __forceinline__ void unpack_chunk(const typename ChunkWord<CB>::type& q, float (&v)[CB / static_cast<int>(sizeof(T))]) {
+    uint32_t w[CB / 4];
+    if constexpr (CB == 16) { w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w; }
+    else if constexpr (CB == 8) { w[0] = q.x; w[1] = q.y; }
+    else { w[0] = q; }
+    if constexpr (sizeof(T) == 4) {
+#pragma unroll
+        for (int e = 0; e < CB / 4; ++e) v[e] = __uint_as_float(w[e]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < CB / 4; ++e) {  // bf16 is the upper half of an fp32
+            v[2 * e] = __uint_as_float(w[e] << 16);
+            v[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
+        }
+    }
+}
+
+// Maximum of a chunk's elements (bf16: on packed pairs, before widening) and its contribution to
+// sum 2^(x L - P) (two-wide FMAs and adds), for chunks of 16, 8 or 4 bytes.
+template <typename T, int CB>
+__device__ __forceinline__ float chunk_max(const typename ChunkWord<CB>::type& q) {
+    uint32_t w[CB / 4];
+    if constexpr (CB == 16) { w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w; }
+    else if constexpr (CB == 8) { w[0] = q.x; w[1] = q.y; }
+    else { w[0] = q; }
+    if constexpr (sizeof(T) == 4) {
+        float m = __uint_as_float(w[0]);
+#pragma unroll
+        for (int e = 1; e < CB / 4; ++e) m = fmaxf(m, __uint_as_float(w[e]));
+        return m;
+    } else {
+        __nv_bfloat162 m = *reinterpret_cast<const __nv_bfloat162*>(&w[0]);
+#pragma unroll
+        for (int e = 1; e < CB / 4; ++e) m = __hmax2(m, *reinterpret_cast<const __nv_bfloat162*>(&w[e]));
+        return fmaxf(__low2float(m), __high2float(m));
+    }
+}
+template <typename T, int CB>
+__device__ __forceinline__ void chunk_sum_exp(const typename ChunkWord<CB>::type& q, F2 l2e, F2 nml, F2& a0, F2& a1) {
+    float v[CB / static_cast<int>(sizeof(T))];
+    unpack_chunk<T, CB>(q, v);
+    constexpr int n = CB / static_cast<int>(sizeof(T));  // 2, 4 or 8 elements
+    pair_sum_exp(v[0], v[1], l2e, nml, a0);
+    if constexpr (n >= 4) pair_sum_exp(v[2], v[3], l2e, nml, a1);
+    if constexpr (n == 8) {
+        pair_sum_exp(v[4], v[5], l2e, nml, a0);
+        pair_sum_exp(v[6], v[7], l2e, nml, a1);
+    }
+}
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst))),
+                 "l"(gsrc)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
+}
+
+// Tiles flow through a ring of kGroupStages buffers filled by asynchronous 16-byte copies (global -> shared, past
+// the registers), one tile ahead of the one being reduced, so every CTA always has loads in flight; two stages
+// rather than three leave room for a third CTA per SM, which is worth more (measured).
+template <typename T, int L, int CB>
+__global__ void __launch_bounds__(kGroupThreads)
+score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
+                        int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0,
+                        int stage_bytes) {
+    constexpr int R = kGroupThreads / L;  // rows per tile = lane groups per CTA
+    constexpr bool VEC = CB > 0;          // rows start on CB-byte boundaries and are whole chunks (base 16-byte aligned)
+    constexpr bool PADDED = CB == 16 && L < 8;
+    constexpr int EPV = VEC ? CB / static_cast<int>(sizeof(T)) : 1;
+    extern __shared__ __align__(16) unsigned char group_smem[];
+    uint32_t* hist_s = reinterpret_cast<uint32_t*>(group_smem);
+    unsigned char* stages = group_smem + kSelBins * sizeof(uint32_t);
+    Hist0 h{hist_s, hist0};
+    h.clear();
+    const int row_bytes = C * static_cast<int>(sizeof(T));
+    const int64_t tiles = (rows + R - 1) / R;
+    const int g = threadIdx.x / L, l = threadIdx.x % L;
+    // 16-byte chunks, L == 4: two rows share a quarter-warp's accesses, so rows are laid out in shared memory with
+    // a pitch of 4 (mod 8) chunks, which puts neighbouring rows four bank groups apart whatever the row length.
+    // (The order in which a row's elements are summed must not depend on where the row sits: copies of a row
+    // have to score the same bits.)
+    const int nchunk = VEC ? row_bytes / (VEC ? CB : 1) : 0;
+    const int pitch_bytes = PADDED ? 16 * (nchunk + ((L - nchunk) & 7)) : row_bytes;
+    const float inv_nchunk = 1.0f / static_cast<float>(nchunk > 0 ? nchunk : 1);
+    const int64_t my_tiles = tiles > blockIdx.x ? (tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+    auto issue = [&](int64_t i) {  // requests this CTA's i-th tile into stage i % kGroupStages
+        if (i < my_tiles) {
+            const int64_t row0 = (blockIdx.x + i * gridDim.x) * R;
+            const int nrows = rows - row0 < R ? static_cast<int>(rows - row0) : R;
+            const uintptr_t b0 = reinterpret_cast<uintptr_t>(logits) + row0 * row_bytes;
+            const int head = VEC ? 0 : static_cast<int>(b0 & 15);
+            const uint4* src = reinterpret_cast<const uint4*>(b0 - head);
+            const int nvec = (head + nrows * row_bytes + 15) >> 4;  // an aligned block that holds a valid byte is safe to read
+            uint4* dst = reinterpret_cast<uint4*>(stages + (i % kGroupStages) * stage_bytes);
+            for (int v = threadIdx.x; v < nvec; v += kGroupThreads) {
+                int d = v;
+                if constexpr (PADDED) {
+                    const int r = __float2int_rz((static_cast<float>(v) + 0.5f) * inv_nchunk);  // v / nchunk, exact here
+                    d = r * (pitch_bytes >> 4) + (v - r * nchunk);
+                }
+                cp_async16(dst + d, src + v);
+            }
+        }
+        cp_async_commit();  // one group per tile slot, also when it is empty: the wait below counts groups
+    };
+    auto label_of = [&](int64_t i) -> int64_t {
+        if (i >= my_tiles) return ignore_index;
+        const int64_t row = (blockIdx.x + i * gridDim.x) * R + g;
+        return row < rows ? labels[row] : ignore_index;
+    };
+
+#pragma unroll
+    for (int i = 0; i < kGroupStages - 1; ++i) issue(i);
+    int64_t y = label_of(0);
+    for (int64_t i = 0; i < my_tiles; ++i) {
+        issue(i + kGroupStages - 1);
+        const int64_t y_next = label_of(i + 1);
+        cp_async_wait<kGroupStages - 1>();
+        __syncthreads();  // everybody's copies of tile i have landed
+        const int64_t row0 = (blockIdx.x + i * gridDim.x) * R;
+        const bool mine = row0 + g < rows;
+        const int head = VEC ? 0 : static_cast<int>((reinterpret_cast<uintptr_t>(logits) + row0 * row_bytes) & 15);
+        unsigned char* buf = stages + (i % kGroupStages) * stage_bytes;
+        const int cls = mine ? label_class(y, C, ignore_index) : 1;
+        T* x = reinterpret_cast<T*>(buf + head + g * pitch_bytes);
+        // the true class stays out of the sum (see loss_without_true_class): its slot is read, then blanked
+        float xy = 0.f;
+        if (cls == 0 && l == 0) {
+            xy = Elem<T>::widen(x[static_cast<int>(y)]);
+            x[static_cast<int>(y)] = Elem<T>::neg_inf_elem();
+        }
+        __syncwarp();
+        float m = -1e30f, s = 0.f;
+        if constexpr (VEC) {
+            using Word = typename ChunkWord<VEC ? CB : 16>::type;
+            const Word* xv = reinterpret_cast<const Word*>(x);
+            const int nch = cls == 0 ? nchunk : 0;  // groups without a row to score run the reductions on nothing
+#pragma unroll 2
+            for (int c = l; c < nch; c += L) m = fmaxf(m, chunk_max<T, VEC ? CB : 16>(xv[c]));
+#pragma unroll
+            for (int o = L / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+            const float P = m * kLog2e;
+            const F2 l2e = pack2(kLog2e, kLog2e), nml = pack2(-P, -P);
+            F2 a0 = pack2(0.f, 0.f), a1 = pack2(0.f, 0.f);
+#pragma unroll 2
+            for (int c = l; c < nch; c += L) chunk_sum_exp<T, VEC ? CB : 16>(xv[c], l2e, nml, a0, a1);
+            float t0, t1, t2, t3;
+            unpack2(a0, t0, t1);
+            unpack2(a1, t2, t3);
+            s = (t0 + t1) + (t2 + t3);
+        } else {
+            const int n = cls == 0 ? C : 0;
+            for (int j = l; j < n; j += L) m = fmaxf(m, Elem<T>::widen(x[j]));
+#pragma unroll
+            for (int o = L / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+            const float P = m * kLog2e;
+            for (int j = l; j < n; j += L) s += ex2(fmaf(Elem<T>::widen(x[j]), kLog2e, -P));
+        }
+#pragma unroll
+        for (int o = L / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+        if (mine && l == 0) {
+            float loss = 0.f;
+            if (cls == 2) {
+                loss = __uint_as_float(0x7FC00000u);
+                atomicAdd(&status->bad_labels, 1);
+            } else if (cls == 0) {
+                loss = loss_without_true_class(m, m * kLog2e, s, xy);
+            }
+            row_loss[row0 + g] = loss;
+            h.add(loss);
+        }
+        __syncthreads();  // the stage may be refilled
+        y = y_next;
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+    h.flush();
 }
 
 // ---------------------------------------------------------------------------
