@@ -228,7 +228,7 @@ def job_throughput(world: int, units_per_rank: float, steps: int, ms: float) -> 
 # profiles/, taken on a scaled-down case and scaled to a full launch by the units processed.  Only for the
 # kernels and workloads that were captured; None elsewhere (and to be reset when a kernel changes).
 NCU_TRAFFIC_BYTES = {
-    ("score", 4): 7.27e9,      # profiles/score_stream_rows_bf16_cfg4.md: 908.8 MB for 128 of 1024 sequences
+    ("score", 4): 7.28e9,      # profiles/score_stream_rows_bf16_cfg4.md: 909.4 MB for 128 of 1024 sequences
     ("aggregate", 4): 4.70e9,  # profiles/aggregate_vec4_cfg4.md: 687.0 MB for 16,000,000 of 109,482,240 parameters
 }
 

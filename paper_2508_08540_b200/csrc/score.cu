@@ -2,16 +2,16 @@
 // data"): softmax cross-entropy per row of the candidate pool, mean over the
 // unmasked tokens of a sample.
 //
-// Every row is evaluated as
-//     m  = max_j x_j
-//     s' = sum over all j except ONE occurrence of the maximum of exp(x_j - m)
-//     l  = (m - x_y) + log1p(s')
-// which is the textbook  (m - x_y) + log(sum_j exp(x_j - m))  with the term that
-// equals exactly 1 taken out of the sum, so that losses near zero keep their
-// relative accuracy in fp32.  exp(x_j - m) is evaluated as
-//     ex2(fma(x_j, L, -fl(m L)))      with L = fl(log2 e),
-// whose argument equals (x_j - m) L + d with d = fma(m, L, -fl(m L)) known
-// exactly; the common factor 2^d is divided out once per row.
+// Every row is evaluated from the sum over the OTHER classes (the true class y is left out):
+//     M = max_{j != y} x_j,   S = sum_{j != y} exp(x_j - M)
+//     x_y >= M:  l = log1p(S exp(M - x_y))
+//     x_y <  M:  l = (M - x_y) + log(S + exp(x_y - M))
+// which equals the textbook  (m - x_y) + log(sum_j exp(x_j - m)),  but adds only positive terms: nothing cancels,
+// so losses near zero (a dominant true class) keep their relative accuracy in fp32, in a single pass and with no
+// comparison per element.  exp(x_j - M) is evaluated as
+//     ex2(fma(x_j, L, -fl(M L)))      with L = fl(log2 e),
+// whose argument equals (x_j - M) L + d with d = fma(M, L, -fl(M L)) known exactly; the common factor 2^d
+// cancels against the same rounded product in the last step (see loss_without_true_class).
 //
 // Row shapes and their kernels (all bound by the bytes of the logits):
 //   tiny rows   (C <= 32)         one thread per row out of a shared-memory tile
@@ -54,24 +54,6 @@ struct Elem<__nv_bfloat16> {
     __device__ static float widen(__nv_bfloat16 v) { return __bfloat162float(v); }
     __device__ static __nv_bfloat16 neg_inf_elem() { return __ushort_as_bfloat16(0xFF80u); }
 };
-
-// Row constants for the exponentials:  ex2(fma(x, L, nml)) = 2^d * exp(x - m).
-struct RowScale {
-    float nml;   // -fl(m L)
-    float corr;  // 2^-d
-    __device__ explicit RowScale(float m) {
-        const float p = m * kLog2e;
-        nml = -p;
-        corr = ex2(-fmaf(m, kLog2e, -p));
-    }
-};
-
-// Final formula.  s_lt: sum of 2^d exp(x_j - m) over the x_j below the maximum;
-// n_max: how many x_j equal the maximum.
-__device__ __forceinline__ float finish_loss(float m, float xy, float s_lt, int n_max, const RowScale& rs) {
-    const float s_excl = fmaf(s_lt, rs.corr, static_cast<float>(n_max - 1));
-    return (m - xy) + log1pf(s_excl);
-}
 
 // The selector's first radix digit, accumulated per CTA in shared memory.
 struct Hist0 {
@@ -243,18 +225,15 @@ score_tiny_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
                 loss = __uint_as_float(0x7FC00000u);
                 atomicAdd(&status->bad_labels, 1);
             } else if (cls == 0) {
-                const float* x = tile + threadIdx.x * pitch;
-                float m = x[0];
-                for (int j = 1; j < C; ++j) m = fmaxf(m, x[j]);
-                const RowScale rs(m);
+                float* x = tile + threadIdx.x * pitch;
+                const float xy = x[static_cast<int>(y)];
+                x[static_cast<int>(y)] = neg_inf();  // the true class stays out of the sum
+                float m = -1e30f;
+                for (int j = 0; j < C; ++j) m = fmaxf(m, x[j]);
+                const float P = m * kLog2e;
                 float s = 0.f;
-                int n_max = 0;
-                for (int j = 0; j < C; ++j) {
-                    const float v = x[j];
-                    if (v < m) s += ex2(fmaf(v, kLog2e, rs.nml));
-                    else ++n_max;
-                }
-                loss = finish_loss(m, x[static_cast<int>(y)], s, n_max, rs);
+                for (int j = 0; j < C; ++j) s += ex2(fmaf(x[j], kLog2e, -P));
+                loss = loss_without_true_class(m, P, s, xy);
             }
             row_loss[row] = loss;
             h.add(loss);
@@ -361,7 +340,6 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
     constexpr int R = kGroupThreads / L;  // rows per tile = lane groups per CTA
     constexpr bool VEC = CB > 0;          // rows start on CB-byte boundaries and are whole chunks (base 16-byte aligned)
     constexpr bool PADDED = CB == 16 && L < 8;
-    constexpr int EPV = VEC ? CB / static_cast<int>(sizeof(T)) : 1;
     extern __shared__ __align__(16) unsigned char group_smem[];
     uint32_t* hist_s = reinterpret_cast<uint32_t*>(group_smem);
     unsigned char* stages = group_smem + kSelBins * sizeof(uint32_t);
@@ -634,7 +612,6 @@ __global__ void __launch_bounds__(kCtaThreads)
 score_huge_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int64_t C,
                        int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0) {
     __shared__ float red_f[kCtaWarps];
-    __shared__ int red_i[kCtaWarps];
     __shared__ uint32_t hist_s[kSelBins];
     Hist0 h{hist_s, hist0};
     h.clear();
@@ -649,37 +626,26 @@ score_huge_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
             if (tid == 0) atomicAdd(&status->bad_labels, 1);
         } else if (cls == 0) {
             const T* x = logits + row * C;
-            float m = neg_inf();
-            for (int64_t j = tid; j < C; j += kCtaThreads) m = fmaxf(m, Elem<T>::widen(x[j]));
+            float m = -1e30f;  // maximum over the other classes (the true class stays out of the sum)
+            for (int64_t j = tid; j < C; j += kCtaThreads)
+                if (j != y) m = fmaxf(m, Elem<T>::widen(x[j]));
             m = warp_max(m);
             if (lane == 0) red_f[warp] = m;
             __syncthreads();
             m = red_f[0];
             for (int w = 1; w < kCtaWarps; ++w) m = fmaxf(m, red_f[w]);
             __syncthreads();
-            const RowScale rs(m);
+            const float P = m * kLog2e;
             float s = 0.f;
-            int n_max = 0;
-            for (int64_t j = tid; j < C; j += kCtaThreads) {
-                const float v = Elem<T>::widen(x[j]);
-                if (v < m) s += ex2(fmaf(v, kLog2e, rs.nml));
-                else ++n_max;
-            }
+            for (int64_t j = tid; j < C; j += kCtaThreads)
+                if (j != y) s += ex2(fmaf(Elem<T>::widen(x[j]), kLog2e, -P));
             s = warp_sum(s);
-            n_max = warp_sum(n_max);
-            if (lane == 0) {
-                red_f[warp] = s;
-                red_i[warp] = n_max;
-            }
+            if (lane == 0) red_f[warp] = s;
             __syncthreads();
             if (tid == 0) {
                 s = red_f[0];
-                n_max = red_i[0];
-                for (int w = 1; w < kCtaWarps; ++w) {
-                    s += red_f[w];
-                    n_max += red_i[w];
-                }
-                loss = finish_loss(m, Elem<T>::widen(x[y]), s, n_max, rs);
+                for (int w = 1; w < kCtaWarps; ++w) s += red_f[w];
+                loss = loss_without_true_class(m, P, s, Elem<T>::widen(x[y]));
             }
         }
         if (tid == 0) {
