@@ -131,6 +131,48 @@ def test_score_closed_forms_and_small_losses(L, oracle):
         assert_losses_close(got, want, C)
 
 
+@pytest.mark.parametrize("C,dtype", [(10, "f32"), (40, "bf16"), (100, "f32"), (102, "bf16"), (500, "f32"), (1000, "bf16"),
+                                     (1500, "f32"), (5000, "bf16"), (30522, "bf16"), (70001, "f32")])
+@pytest.mark.parametrize("off", [0, 1, 3])
+def test_score_true_class_anywhere_confident_or_not(L, oracle, C, dtype, off):
+    """The true class is the one term every kernel leaves out of its sum: put it at the row's ends (the partial
+    vectors of unaligned rows), next to them and in the middle, as the dominant class, as a runner-up, tied with the
+    maximum, and far below it."""
+    ys = sorted({0, 1, 2, 3, 7, 8, C // 2, C - 9, C - 8, C - 4, C - 3, C - 2, C - 1} & set(range(C)))
+    rows, labels = [], []
+    rng = np.random.default_rng(C + off)
+    for y in ys:
+        for kind in range(4):
+            r = rng.normal(0, 2, C).astype(np.float32)
+            top = float(r.max())
+            if kind == 0:
+                r[y] = top + 12.0      # dominant: a loss of about 1e-4, relative accuracy needed
+            elif kind == 1:
+                r[y] = top - 0.5       # runner-up
+            elif kind == 2:
+                r[y] = top             # tied with the maximum (unless y already is the maximum)
+            else:
+                r[y] = top - 30.0      # hopeless
+            rows.append(r)
+            labels.append(y)
+    x = np.stack(rows)
+    y = np.array(labels, dtype=np.int64)
+    if dtype == "bf16":
+        x = wl.f32_to_bf16_bits(x)
+    want, bad = oracle.score(x, y)
+    assert bad == 0
+    flat = dev_logits(x).reshape(-1)
+    buf = torch.zeros(flat.numel() + 8, dtype=flat.dtype, device="cuda")
+    buf[off:off + flat.numel()] = flat
+    got = L.score_losses(buf[off:off + flat.numel()].view(len(rows), C), torch.from_numpy(y).cuda()).cpu().numpy()
+    assert_losses_close(got, want, C)
+    # dominant rows: the cancellation-free closed form, to 1e-5 relative whatever the oracle's own floor
+    xd = (wl.bf16_bits_to_f32(x) if dtype == "bf16" else x).astype(np.float64)
+    dom = np.arange(0, len(rows), 4)
+    others = np.array([np.exp(np.delete(xd[i], y[i]) - xd[i, y[i]]).sum() for i in dom])
+    np.testing.assert_allclose(got[dom], np.log1p(others), rtol=1e-5, atol=0)
+
+
 @pytest.mark.parametrize("C,dtype", [(10, "f32"), (100, "f32"), (5000, "bf16")])
 def test_score_masks_bad_labels_and_sequences(L, oracle, C, dtype):
     N, T = 9, 6
