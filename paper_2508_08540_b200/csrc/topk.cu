@@ -393,6 +393,8 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
     __shared__ uint32_t counters[kWarps][kSortBins];
     __shared__ uint32_t base_s[kSortBins];
     __shared__ uint32_t tot_s[kSortBins];
+    constexpr int kParts = kSortThreads / kSortBins;
+    __shared__ uint32_t part_tot[kParts][kSortBins], part_bef[kParts][kSortBins];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t tiles = (k + kTile - 1) / kTile;
     const int shift = 8 * pass;
@@ -400,21 +402,26 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
     for (uint32_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
         // where each digit's run starts for this tile: all entries of earlier digits, plus
         // this digit's entries in earlier tiles
-        uint32_t before = 0;
-        if (tid < kSortBins) {
-            uint32_t total = 0;
-            for (uint32_t t0 = 0; t0 < tiles; t0 += 8) {
+        // (four threads per digit, each over a quarter of the tiles: the chain of dependent loads is what a
+        // pass with many tiles waits for)
+        {
+            const int d = tid & (kSortBins - 1), q = tid / kSortBins;
+            const uint32_t per = (tiles + kParts - 1) / kParts;
+            const uint32_t t_lo = q * per, t_hi = min(tiles, t_lo + per);
+            uint32_t total = 0, bef = 0;
+            for (uint32_t t0 = t_lo; t0 < t_hi; t0 += 8) {
                 uint32_t c[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u)  // eight independent loads in flight
-                    c[u] = t0 + u < tiles ? __ldcg(tile_hist + (t0 + u) * kSortBins + tid) : 0u;
+                    c[u] = t0 + u < t_hi ? __ldcg(tile_hist + (t0 + u) * kSortBins + d) : 0u;
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     total += c[u];
-                    before += t0 + u < tile ? c[u] : 0u;
+                    bef += t0 + u < tile ? c[u] : 0u;
                 }
             }
-            tot_s[tid] = total;
+            part_tot[q][d] = total;
+            part_bef[q][d] = bef;
         }
 #pragma unroll
         for (int i = 0; i < kWarps * kSortBins / kSortThreads; ++i) (&counters[0][0])[i * kSortThreads + tid] = 0;
@@ -426,6 +433,17 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
             const uint32_t e = first + rd * 32 + lane;
             key[rd] = e < k ? __ldcg(keys_in + e) : 0u;
             idx[rd] = e < k ? __ldcg(idx_in + e) : 0;
+        }
+        __syncthreads();
+        uint32_t before = 0;
+        if (tid < kSortBins) {
+            uint32_t total = 0;
+#pragma unroll
+            for (int q = 0; q < kParts; ++q) {
+                total += part_tot[q][tid];
+                before += part_bef[q][tid];
+            }
+            tot_s[tid] = total;
         }
         __syncthreads();
         if (warp == 0) {  // exclusive scan of the 256 digit totals, eight per lane
