@@ -305,6 +305,46 @@ __device__ __forceinline__ float chunk_max(const typename ChunkWord<CB>::type& q
         return fmaxf(__low2float(m), __high2float(m));
     }
 }
+// A chunk of -inf elements, and a running maximum over chunks (bf16: on packed pairs, widened once at the end).
+template <typename T, int CB>
+__device__ __forceinline__ typename ChunkWord<CB>::type chunk_fill() {
+    constexpr uint32_t f = sizeof(T) == 4 ? 0xFF800000u : 0xFF80FF80u;
+    if constexpr (CB == 16) return make_uint4(f, f, f, f);
+    else if constexpr (CB == 8) return make_uint2(f, f);
+    else return f;
+}
+template <typename T>
+struct ChunkMax;
+template <>
+struct ChunkMax<float> {
+    float m;
+    __device__ ChunkMax() : m(neg_inf()) {}
+    __device__ __forceinline__ void word(uint32_t w) { m = fmaxf(m, __uint_as_float(w)); }
+    template <int CB>
+    __device__ __forceinline__ void add(const typename ChunkWord<CB>::type& q) {
+        if constexpr (CB == 16) { word(q.x); word(q.y); word(q.z); word(q.w); }
+        else if constexpr (CB == 8) { word(q.x); word(q.y); }
+        else word(q);
+    }
+    __device__ __forceinline__ float get() const { return m; }
+};
+template <>
+struct ChunkMax<__nv_bfloat16> {
+    uint32_t m;
+    __device__ ChunkMax() : m(0xFF80FF80u) {}
+    __device__ __forceinline__ void word(uint32_t w) {
+        const __nv_bfloat162 r = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&m), *reinterpret_cast<const __nv_bfloat162*>(&w));
+        m = *reinterpret_cast<const uint32_t*>(&r);
+    }
+    template <int CB>
+    __device__ __forceinline__ void add(const typename ChunkWord<CB>::type& q) {
+        if constexpr (CB == 16) { word(q.x); word(q.y); word(q.z); word(q.w); }
+        else if constexpr (CB == 8) { word(q.x); word(q.y); }
+        else word(q);
+    }
+    __device__ __forceinline__ float get() const { return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u)); }
+};
+
 template <typename T, int CB>
 __device__ __forceinline__ void chunk_sum_exp(const typename ChunkWord<CB>::type& q, F2 l2e, F2 nml, F2& a0, F2& a1) {
     float v[CB / static_cast<int>(sizeof(T))];
@@ -333,7 +373,7 @@ __device__ __forceinline__ void cp_async_wait() {
 // the registers), one tile ahead of the one being reduced, so every CTA always has loads in flight; two stages
 // rather than three leave room for a third CTA per SM, which is worth more (measured).
 template <typename T, int L, int CB>
-__global__ void __launch_bounds__(kGroupThreads)
+__global__ void __launch_bounds__(kGroupThreads, 4)
 score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
                         int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0,
                         int stage_bytes) {
@@ -405,10 +445,44 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
         }
         __syncwarp();
         float m = -1e30f, s = 0.f;
-        if constexpr (VEC) {
-            using Word = typename ChunkWord<VEC ? CB : 16>::type;
+        if constexpr (VEC && L >= 8) {
+            // A lane's share of a row is at most 128 bytes (rows of up to 512, 1024, 2048 bytes over 4, 8, 16
+            // lanes): it is read from shared memory once, into registers, and both passes run from there, fully
+            // unrolled.  Round i (chunks i L .. i L + L - 1) is skipped by the whole warp once it is past the row.
+            constexpr int CBV = VEC ? CB : 16;
+            constexpr int kMaxCh = 128 / CBV;
+            using Word = typename ChunkWord<CBV>::type;
             const Word* xv = reinterpret_cast<const Word*>(x);
             const int nch = cls == 0 ? nchunk : 0;  // groups without a row to score run the reductions on nothing
+            Word w[kMaxCh];
+            ChunkMax<T> cm;
+#pragma unroll
+            for (int i = 0; i < kMaxCh; ++i) {
+                if (i * L < nchunk) {  // the same for every thread of the CTA
+                    const int c = l + i * L;
+                    w[i] = c < nch ? xv[c] : chunk_fill<T, CBV>();
+                    cm.template add<CBV>(w[i]);
+                }
+            }
+            m = fmaxf(m, cm.get());
+#pragma unroll
+            for (int o = L / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+            const float P = m * kLog2e;
+            const F2 l2e = pack2(kLog2e, kLog2e), nml = pack2(-P, -P);
+            F2 a0 = pack2(0.f, 0.f), a1 = pack2(0.f, 0.f);
+#pragma unroll
+            for (int i = 0; i < kMaxCh; ++i)
+                if (i * L < nchunk) chunk_sum_exp<T, CBV>(w[i], l2e, nml, a0, a1);
+            float t0, t1, t2, t3;
+            unpack2(a0, t0, t1);
+            unpack2(a1, t2, t3);
+            s = (t0 + t1) + (t2 + t3);
+        } else if constexpr (VEC) {
+            // short rows (4 lanes per row): a few chunks per lane, plain loops (measured faster here than the
+            // unrolled register copy above, whose fixed cost these rows do not repay)
+            using Word = typename ChunkWord<VEC ? CB : 16>::type;
+            const Word* xv = reinterpret_cast<const Word*>(x);
+            const int nch = cls == 0 ? nchunk : 0;
 #pragma unroll 2
             for (int c = l; c < nch; c += L) m = fmaxf(m, chunk_max<T, VEC ? CB : 16>(xv[c]));
 #pragma unroll
