@@ -136,7 +136,7 @@ LSGD_API lsgd_status lsgd_topk_select(const float* losses, int64_t N, int64_t k,
  * device allocator of their own.  The paper has no counterpart to this entry
  * point; it is a convenience of this library.
  *
- * The scratch is a fixed array of about 4.3 MiB inside the library's device
+ * The scratch is a fixed array of about 4.5 MiB inside the library's device
  * image (every GPU that loads the library holds it until the process ends), so
  * the pool is limited to N <= LSGD_STATIC_TOPK_MAX_N; a larger N returns
  * LSGD_ERR_UNSUPPORTED and nothing is launched.  Arguments, result and order are

@@ -28,13 +28,24 @@
 
 namespace lsgd {
 
+// The sort of the selected pairs works on tiles of 1024 entries when k is small (more, shorter CTAs: the pass is
+// latency-bound) and of kTile entries otherwise (fewer tiles to prefix over).
+constexpr int64_t kSmallSortK = 131072;
+static int sort_tile_shift(int64_t k) { return k <= kSmallSortK ? 10 : 12; }
+static size_t sort_tiles(int64_t k) { return static_cast<size_t>((k + (int64_t{1} << sort_tile_shift(k)) - 1) >> sort_tile_shift(k)); }
+// Tiles reserved for the digit counts: an upper bound of sort_tiles() that grows with k, so that a workspace sized
+// for k also serves every smaller k.
+static size_t sort_tiles_bound(int64_t k) {
+    const size_t small = static_cast<size_t>((std::min<int64_t>(k, kSmallSortK) + 1023) / 1024);
+    return std::max(small, static_cast<size_t>((k + kTile - 1) / kTile));
+}
+
 size_t topk_workspace_bytes(int64_t N, int64_t k) {
     if (N < 0 || k < 0 || k > N) return 0;
     const size_t tiles_n = static_cast<size_t>((N + kTile - 1) / kTile);
-    const size_t tiles_k = static_cast<size_t>((k + kTile - 1) / kTile);
     size_t b = sizeof(StatusBlock);
     b += align_up(sizeof(uint32_t) * kSelPasses * kSelBins);
-    b += align_up(sizeof(uint32_t) * 4 * tiles_k * kSortBins);
+    b += align_up(sizeof(uint32_t) * 4 * sort_tiles_bound(k) * kSortBins);
     b += align_up(sizeof(uint32_t) * 2 * tiles_n);
     b += 4 * align_up(sizeof(uint32_t) * static_cast<size_t>(k));
     return b;
@@ -42,14 +53,12 @@ size_t topk_workspace_bytes(int64_t N, int64_t k) {
 
 // Bytes at the start of the workspace that one memset must clear before a call.
 static size_t topk_zero_bytes(int64_t k) {
-    const size_t tiles_k = static_cast<size_t>((k + kTile - 1) / kTile);
     return sizeof(StatusBlock) + align_up(sizeof(uint32_t) * kSelPasses * kSelBins) +
-           align_up(sizeof(uint32_t) * 4 * tiles_k * kSortBins);
+           align_up(sizeof(uint32_t) * 4 * sort_tiles_bound(k) * kSortBins);
 }
 
 TopkWorkspace carve_topk(void* ws, int64_t N, int64_t k) {
     const size_t tiles_n = static_cast<size_t>((N + kTile - 1) / kTile);
-    const size_t tiles_k = static_cast<size_t>((k + kTile - 1) / kTile);
     unsigned char* p = static_cast<unsigned char*>(ws);
     TopkWorkspace w;
     w.status = reinterpret_cast<StatusBlock*>(p);
@@ -57,7 +66,7 @@ TopkWorkspace carve_topk(void* ws, int64_t N, int64_t k) {
     w.hist = reinterpret_cast<uint32_t*>(p);
     p += align_up(sizeof(uint32_t) * kSelPasses * kSelBins);
     w.tile_hist = reinterpret_cast<uint32_t*>(p);
-    p += align_up(sizeof(uint32_t) * 4 * tiles_k * kSortBins);
+    p += align_up(sizeof(uint32_t) * 4 * sort_tiles_bound(k) * kSortBins);
     w.tile_counts = reinterpret_cast<uint32_t*>(p);
     p += align_up(sizeof(uint32_t) * 2 * tiles_n);
     const size_t kb = align_up(sizeof(uint32_t) * static_cast<size_t>(k));
@@ -299,7 +308,8 @@ template <bool DIRECT>
 __global__ void __launch_bounds__(kThreads)
 select_emit_kernel(const float* __restrict__ losses, int64_t N, const StatusBlock* status,
                    const uint32_t* tile_counts, int32_t* __restrict__ out_idx,
-                   float* __restrict__ out_vals, uint32_t* __restrict__ out_keys, uint32_t* __restrict__ tile_hist) {
+                   float* __restrict__ out_vals, uint32_t* __restrict__ out_keys, uint32_t* __restrict__ tile_hist,
+                   int sort_shift) {
     __shared__ uint32_t scratch[kThreads / 32 + 1];
     __shared__ uint32_t pre[2];
     grid_dependency_wait();
@@ -350,7 +360,7 @@ select_emit_kernel(const float* __restrict__ losses, int64_t N, const StatusBloc
                 } else {
                     out_idx[pos] = static_cast<int32_t>(j);
                     out_keys[pos] = key[i];
-                    atomicAdd(&tile_hist[(pos / kTile) * kSortBins + (255u - (key[i] & 0xFFu))], 1u);
+                    atomicAdd(&tile_hist[(pos >> sort_shift) * kSortBins + (255u - (key[i] & 0xFFu))], 1u);
                 }
             }
             gt_run += above;
@@ -381,14 +391,16 @@ __device__ __forceinline__ uint32_t match_digit8(uint32_t d, bool live) {
 // tile is spread over 32 warps: four ranking rounds per warp instead of sixteen.
 constexpr int kSortThreads = 1024;
 
-template <bool LAST>
+template <bool LAST, int kRounds>  // kRounds rounds of 32 consecutive entries per warp: tiles of 1024 kRounds entries
 __global__ void __launch_bounds__(kSortThreads)
 sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restrict__ idx_in, uint32_t k, int pass,
                     const uint32_t* __restrict__ tile_hist, uint32_t* __restrict__ keys_out,
                     int32_t* __restrict__ idx_out, uint32_t* __restrict__ next_hist,
                     const float* __restrict__ losses, float* __restrict__ out_vals) {
     constexpr int kWarps = kSortThreads / 32;
-    constexpr int kRounds = kTile / kSortThreads;  // rounds of 32 consecutive entries per warp
+    constexpr uint32_t kSortTile = kSortThreads * kRounds;
+    constexpr int kSortShift = kRounds == 1 ? 10 : 12;
+    static_assert(kRounds == 1 || kRounds == 4, "tiles of 1024 or 4096 entries");
     static_assert(kSortBins == 256 && kSortThreads >= kSortBins, "one thread per digit in the scans");
     __shared__ uint32_t counters[kWarps][kSortBins];
     __shared__ uint32_t base_s[kSortBins];
@@ -396,7 +408,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
     constexpr int kParts = kSortThreads / kSortBins;
     __shared__ uint32_t part_tot[kParts][kSortBins], part_bef[kParts][kSortBins];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t tiles = (k + kTile - 1) / kTile;
+    const uint32_t tiles = (k + kSortTile - 1) / kSortTile;
     const int shift = 8 * pass;
     grid_dependency_wait();
     for (uint32_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
@@ -427,7 +439,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
         for (int i = 0; i < kWarps * kSortBins / kSortThreads; ++i) (&counters[0][0])[i * kSortThreads + tid] = 0;
         uint32_t key[kRounds], rank[kRounds];
         int32_t idx[kRounds];
-        const uint32_t first = tile * kTile + warp * (kRounds * 32);
+        const uint32_t first = tile * kSortTile + warp * (kRounds * 32);
 #pragma unroll
         for (int rd = 0; rd < kRounds; ++rd) {  // all loads first: they are independent
             const uint32_t e = first + rd * 32 + lane;
@@ -516,7 +528,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
                 const uint32_t nd = 255u - ((key[rd] >> (shift + 8)) & 0xFFu);
                 const uint32_t peers = match_digit8(nd, live);
                 const int leader = live ? __ffs(peers) - 1 : lane;
-                const uint32_t t = pos / kTile;
+                const uint32_t t = pos >> kSortShift;
                 const bool with_leader = t == __shfl_sync(0xFFFFFFFFu, t, leader);  // same destination tile as the leader
                 const uint32_t same = __ballot_sync(0xFFFFFFFFu, live && with_leader);
                 if (live) {
@@ -619,19 +631,25 @@ cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order or
     if (e != cudaSuccess) return e;
     if (order == LSGD_ORDER_INDEX_ASC)
         return launch_dependent(select_emit_kernel<true>, grid_n, kThreads, s, losses, N, ws.status, ws.tile_counts,
-                                out_idx, out_vals, nullptr, nullptr);
-    const int64_t tiles_k = (k + kTile - 1) / kTile;
-    const size_t th = static_cast<size_t>(tiles_k) * kSortBins;
+                                out_idx, out_vals, nullptr, nullptr, 12);
+    const int sort_shift = sort_tile_shift(k);
+    const int64_t tiles_k = static_cast<int64_t>(sort_tiles(k));
+    const size_t th = sort_tiles_bound(k) * kSortBins;  // digit counts of one pass
     e = launch_dependent(select_emit_kernel<false>, grid_n, kThreads, s, losses, N, ws.status, ws.tile_counts, ws.idx[0],
-                         nullptr, ws.keys[0], ws.tile_hist);
+                         nullptr, ws.keys[0], ws.tile_hist, sort_shift);
     const int grid_k = static_cast<int>(std::min<int64_t>(tiles_k, static_cast<int64_t>(sm_count()) * 2));
-    for (int pass = 0; pass < 3 && e == cudaSuccess; ++pass)
-        e = launch_dependent(sort_scatter_kernel<false>, grid_k, kSortThreads, s, ws.keys[pass & 1], ws.idx[pass & 1], kk, pass,
-                             ws.tile_hist + pass * th, ws.keys[(pass + 1) & 1], ws.idx[(pass + 1) & 1],
-                             ws.tile_hist + (pass + 1) * th, nullptr, nullptr);
-    if (e != cudaSuccess) return e;
-    return launch_dependent(sort_scatter_kernel<true>, grid_k, kSortThreads, s, ws.keys[1], ws.idx[1], kk, 3,
-                            ws.tile_hist + 3 * th, nullptr, out_idx, nullptr, losses, out_vals);
+    auto pass_kernel = [&](auto mid, auto last) {
+        for (int pass = 0; pass < 3 && e == cudaSuccess; ++pass)
+            e = launch_dependent(mid, grid_k, kSortThreads, s, ws.keys[pass & 1], ws.idx[pass & 1], kk, pass,
+                                 ws.tile_hist + pass * th, ws.keys[(pass + 1) & 1], ws.idx[(pass + 1) & 1],
+                                 ws.tile_hist + (pass + 1) * th, nullptr, nullptr);
+        if (e != cudaSuccess) return;
+        e = launch_dependent(last, grid_k, kSortThreads, s, ws.keys[1], ws.idx[1], kk, 3, ws.tile_hist + 3 * th, nullptr,
+                             out_idx, nullptr, losses, out_vals);
+    };
+    if (sort_shift == 10) pass_kernel(sort_scatter_kernel<false, 1>, sort_scatter_kernel<true, 1>);
+    else pass_kernel(sort_scatter_kernel<false, 4>, sort_scatter_kernel<true, 4>);
+    return e;
 }
 
 }  // namespace lsgd
