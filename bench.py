@@ -339,7 +339,8 @@ def run_gpu(args, cfg):
         torch.cuda.synchronize()
         warm = {"score_topk_ms": float(np.median([e[0].elapsed_time(e[1]) for e in w_ev])),
                 "aggregate_ms": float(np.median([e[1].elapsed_time(e[2]) for e in w_ev])),
-                "note": "same step without the L2 flush (inputs may be L2-resident); median of 20"}
+                "note": "same step without the L2 flush (inputs may be L2-resident); median of 20; with nothing between the "
+                        "steps the host's enqueue rate, not the device, bounds steps shorter than about 60 us"}
 
     # ---- end to end: inputs from pinned host memory, results back to the host, every step
     e2e_steps = max(1, min(args.steps, 5 if cfg.logit_bytes > (1 << 30) else 20))
