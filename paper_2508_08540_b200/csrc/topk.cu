@@ -557,7 +557,36 @@ small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int
         ck[i] = i < n ? (static_cast<unsigned long long>(loss_key(losses[i])) << 32) | (0xFFFFFFFFu - static_cast<uint32_t>(i))
                       : 0ull;
     __syncthreads();
-    for (int size = 2; size <= n2; size <<= 1)
+    if (n2 <= kSmallThreads) {
+        // One entry per thread, in a register: steps with stride < 32 exchange by shuffle, the wider ones through
+        // shared memory.  Entry i keeps the larger of the pair if it is the lower index of a descending run (or the
+        // upper index of an ascending one).
+        const int i = threadIdx.x;
+        unsigned long long v = i < n2 ? ck[i] : 0ull;
+        for (int size = 2; size <= n2; size <<= 1) {
+            const bool desc = (i & size) == 0;
+            for (int stride = size >> 1; stride > 0; stride >>= 1) {
+                unsigned long long pv;
+                if (stride >= 32) {
+                    __syncthreads();  // the previous round's reads are done
+                    if (i < n2) ck[i] = v;
+                    __syncthreads();
+                    pv = i < n2 ? ck[i ^ stride] : 0ull;
+                } else {
+                    pv = __shfl_xor_sync(0xFFFFFFFFu, v, stride);
+                }
+                const bool take_max = ((i & stride) == 0) == desc;
+                v = take_max ? (v > pv ? v : pv) : (v < pv ? v : pv);
+            }
+        }
+        __syncthreads();
+        if (i < n2) ck[i] = v;
+        __syncthreads();
+    } else {
+    // Pair t of a step with stride <= 32 lies in the 64 entries [64 (t / 32), 64 (t / 32) + 64), which only the warp
+    // that owns pairs 32 (t / 32) .. + 31 touches in that step and in all the narrower ones after it: those steps
+    // need a warp barrier only, and the CTA-wide one once per size.
+    for (int size = 2; size <= n2; size <<= 1) {
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
             for (int t = threadIdx.x; t < (n2 >> 1); t += kSmallThreads) {
                 const int lo = ((t / stride) * stride << 1) + (t % stride);
@@ -569,8 +598,12 @@ small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int
                     ck[hi] = a;
                 }
             }
-            __syncthreads();
+            if (stride > 32) __syncthreads();
+            else if (stride > 1) __syncwarp();
         }
+        __syncthreads();
+    }
+    }
     grid_launch_dependents();
     if (order == LSGD_ORDER_LOSS_DESC) {
         for (int j = threadIdx.x; j < k; j += kSmallThreads) {
