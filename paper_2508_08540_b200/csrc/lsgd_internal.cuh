@@ -37,7 +37,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 constexpr int kSelPasses = 3;
 constexpr int kSelBins = 2048;            // 11-bit digits (the last digit uses 1024 of them)
 constexpr int kTile = 4096;               // elements per CTA in the count / emit / sort kernels
-constexpr int kSmallN = 4096;             // pools up to this size are sorted by one CTA in shared memory
+constexpr int kSmallN = 1024;             // pools up to this size are sorted by one CTA, one entry per thread
 constexpr int kSortBins = 256;            // 8-bit digits of the stable LSD sort of the selected pairs
 
 struct TopkWorkspace {       // device pointers carved out of the caller's workspace

@@ -541,8 +541,8 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
     }
 }
 
-// Small pools: one CTA sorts all N composite keys (key, ~index) in shared memory
-// with a bitonic network; the first k are the selection in loss-descending order.
+// Small pools: one CTA sorts all N composite keys (key, ~index), one per thread, with a
+// bitonic network; the first k are the selection in loss-descending order.
 constexpr int kSmallThreads = 1024;
 
 __global__ void __launch_bounds__(kSmallThreads)
@@ -557,7 +557,8 @@ small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int
         ck[i] = i < n ? (static_cast<unsigned long long>(loss_key(losses[i])) << 32) | (0xFFFFFFFFu - static_cast<uint32_t>(i))
                       : 0ull;
     __syncthreads();
-    if (n2 <= kSmallThreads) {
+    static_assert(kSmallN <= kSmallThreads, "one entry per thread");
+    {
         // One entry per thread, in a register: steps with stride < 32 exchange by shuffle, the wider ones through
         // shared memory.  Entry i keeps the larger of the pair if it is the lower index of a descending run (or the
         // upper index of an ascending one).
@@ -582,27 +583,6 @@ small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int
         __syncthreads();
         if (i < n2) ck[i] = v;
         __syncthreads();
-    } else {
-    // Pair t of a step with stride <= 32 lies in the 64 entries [64 (t / 32), 64 (t / 32) + 64), which only the warp
-    // that owns pairs 32 (t / 32) .. + 31 touches in that step and in all the narrower ones after it: those steps
-    // need a warp barrier only, and the CTA-wide one once per size.
-    for (int size = 2; size <= n2; size <<= 1) {
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            for (int t = threadIdx.x; t < (n2 >> 1); t += kSmallThreads) {
-                const int lo = ((t / stride) * stride << 1) + (t % stride);
-                const int hi = lo + stride;
-                const bool desc = ((lo & size) == 0);  // this half of the network sorts descending
-                const unsigned long long a = ck[lo], b = ck[hi];
-                if ((a < b) == desc) {
-                    ck[lo] = b;
-                    ck[hi] = a;
-                }
-            }
-            if (stride > 32) __syncthreads();
-            else if (stride > 1) __syncwarp();
-        }
-        __syncthreads();
-    }
     }
     grid_launch_dependents();
     if (order == LSGD_ORDER_LOSS_DESC) {
@@ -615,7 +595,7 @@ small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int
     }
     // index-ascending: an entry is selected iff its composite key is >= the k-th largest
     const unsigned long long cut = ck[k - 1];
-    constexpr int kPer = kSmallN / kSmallThreads;  // 4 consecutive indices per thread
+    constexpr int kPer = 1;  // one index per thread
     const int base = threadIdx.x * kPer;
     bool sel[kPer];
     uint32_t mine = 0;
