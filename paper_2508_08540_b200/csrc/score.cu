@@ -541,21 +541,6 @@ constexpr int kStreamU = 4;                       // vectors (16 bytes) per lane
 constexpr int kStreamMaxRowBytes = 256 * 1024;
 
 template <typename T>
-__device__ __forceinline__ void widen_vector(const uint4& q, float (&v)[Elem<T>::kPerVec]) {
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-    if constexpr (Elem<T>::kPerVec == 4) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) v[e] = __uint_as_float(w[e]);
-    } else {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            v[2 * e] = __uint_as_float(w[e] << 16);
-            v[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
-        }
-    }
-}
-
-template <typename T>
 __global__ void __launch_bounds__(kStreamThreads)
 score_stream_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
                          int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0,
