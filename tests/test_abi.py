@@ -170,3 +170,23 @@ def test_aggregate_round_argument_errors(L):
     assert f(ctypes.cast(odd, ctypes.c_void_p), 1, wp, 1, 16, None, far, 0, None) == L.ERR_ALIGNMENT
     twice = (ctypes.c_void_p * 2)(0x10000, 0x10000)
     assert f(ctypes.cast(twice, ctypes.c_void_p), 0, w2, 2, 16, None, far, 1, None) == L.ERR_INVALID_ARG  # broadcast into aliased replicas
+
+
+def test_binding_fails_loudly_without_the_library(tmp_path):
+    """There is no CPU or library fallback: without liblsgd.so every entry point raises."""
+    import subprocess
+    import sys
+
+    code = (
+        "import sys; sys.path.insert(0, %r)\n"
+        "from paper_2508_08540_b200 import lsgd\n"
+        "lsgd.LIB_PATH = %r\n"
+        "try:\n"
+        "    lsgd.weights_from_steps([1, 2])\n"
+        "except ImportError as e:\n"
+        "    print('raised', 'missing' in str(e))\n"
+        "else:\n"
+        "    print('no error')\n"
+    ) % (ROOT, str(tmp_path / "liblsgd.so"))
+    out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=300)
+    assert out.stdout.strip() == "raised True", out.stdout + out.stderr
