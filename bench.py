@@ -492,6 +492,7 @@ def launches_per_step(cfg) -> int:
 
 
 SWEEP_SHAPES = (  # rows, classes, dtype: one row shape per scorer kernel and regime, each pool larger than L2
+    (20_000_000, 10, "f32"), (12_000_000, 32, "bf16"),
     (8_000_000, 48, "f32"), (5_000_000, 100, "f32"), (4_000_000, 200, "f32"), (2_000_000, 500, "f32"),
     (1_281_167, 1000, "f32"), (640_000, 2000, "f32"), (150_000, 8000, "f32"), (40_000, 30522, "f32"),
     (6_000_000, 100, "bf16"), (3_000_000, 300, "bf16"), (2_000_000, 1000, "bf16"), (1_000_000, 2000, "bf16"),

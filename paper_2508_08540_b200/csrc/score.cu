@@ -204,6 +204,7 @@ score_tiny_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
     Hist0 h{hist_s, hist0};
     h.clear();
     const int pitch = C | 1;  // odd pitch: conflict-free row reads
+    const int step_r = kTinyThreads / C, step_c = kTinyThreads - step_r * C;
     const int64_t tiles = (rows + kTinyThreads - 1) / kTinyThreads;
     for (int64_t t = blockIdx.x; t < tiles; t += gridDim.x) {
         const int64_t row0 = t * kTinyThreads;
@@ -211,9 +212,17 @@ score_tiny_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
         const T* src = logits + row0 * C;
         const int n = nrows * C;
         __syncthreads();
-        for (int i = threadIdx.x; i < n; i += kTinyThreads) {
-            const int r = i / C;
-            tile[r * pitch + (i - r * C)] = Elem<T>::widen(src[i]);
+        {   // element i = r C + c; i advances by the CTA size, (r, c) by its quotient and remainder
+            int r = threadIdx.x / C, c = threadIdx.x - r * C;
+            for (int i = threadIdx.x; i < n; i += kTinyThreads) {
+                tile[r * pitch + c] = Elem<T>::widen(src[i]);
+                r += step_r;
+                c += step_c;
+                if (c >= C) {
+                    c -= C;
+                    ++r;
+                }
+            }
         }
         __syncthreads();
         if (threadIdx.x < nrows) {
