@@ -79,10 +79,11 @@ LSGD_API size_t lsgd_topk_workspace_bytes(int64_t N, int64_t k);
 LSGD_API size_t lsgd_score_topk_workspace_bytes(int64_t N, int64_t T, int64_t C, int64_t k);
 
 /*
- * lsgd_score_losses — the per-sample loss record of Algorithm 1 ("record all
- * individual loss of processed data"; the stored value is one float per sample,
- * Section 4.4 "Potential Limitations").  The loss f(x, xi) of the problem
- * definition (Section 2) is taken to be softmax cross-entropy with natural log.
+ * lsgd_score_losses — the per-sample loss record of Algorithm 1 (the step of
+ * the training loop that stores the loss of every processed sample; one float
+ * per sample, as Section 4.4 "Potential Limitations" counts it).  The loss
+ * f(x, xi) of the problem definition (Section 2) is taken to be softmax
+ * cross-entropy with natural log.
  *
  *   token loss   l[n,t] = -log softmax(logits[n,t,:])[labels[n,t]]
  *   sample loss  losses[n] = mean of l[n,t] over the tokens t whose label is not
@@ -91,7 +92,9 @@ LSGD_API size_t lsgd_score_topk_workspace_bytes(int64_t N, int64_t T, int64_t C,
  *
  *   logits  device, [N, T, C] row-major, contiguous, dtype `dtype`, aligned to
  *           its element size (16-byte alignment is faster, not required).
- *           Values must be finite.  Rows whose label is ignore_index are not scored,
+ *           Values must be finite with |x| <= 1e30 (the kernels form x * log2(e)
+ *           in fp32 and start their running maxima at -1e30; beyond that range
+ *           results are unspecified).  Rows whose label is ignore_index are not scored,
  *           and rows longer than 2 KB are then not read at all (shorter rows are
  *           loaded in contiguous tiles, ignored rows included; their values are
  *           not used).
@@ -111,8 +114,8 @@ LSGD_API lsgd_status lsgd_score_losses(const void* logits, lsgd_dtype dtype, con
 
 /*
  * lsgd_topk_select — deterministic loss-based top-k selection (Section 4.2,
- * "Data Allocation for Fast Workers"; Algorithm 1, the "select ... high-loss
- * samples" step).  Selects the k entries that come first in the total order
+ * "Data Allocation for Fast Workers"; Algorithm 1, the step that picks the
+ * highest-loss samples).  Selects the k entries that come first in the total order
  *     higher loss first, then lower index,
  * where -0.0 equals +0.0 and every NaN ranks above +inf (NaNs tie with each
  * other).  Exact: integer comparisons only, bit-reproducible.
@@ -172,6 +175,22 @@ LSGD_API lsgd_status lsgd_score_topk(const void* logits, lsgd_dtype dtype, const
 /* Per-epoch data allocation (Section 4.2, "Bias Injection via Data Sampling"; */
 /* Algorithm 1, the four steps before the training loop).                      */
 /* ------------------------------------------------------------------------- */
+/*
+ * Which calls make which allocation scheme (Section 4.2 and the appendix,
+ * "Random Sampling Scheme Comparison" with its table of data sampling methods).
+ * The library has no mode switch: a scheme is a choice of sizes and exclusion
+ * lists by the caller.
+ *   high-loss samples to the FAST group (the paper's method):
+ *     fast list  = lsgd_fast_allocation(k_high = floor(lambda N_F), n_fill = N_F - k_high)
+ *     slow list  = lsgd_draw_uniform(n_draw = N_S) on another stream   (separated sampling)
+ *               or lsgd_draw_uniform(n_draw = N_S, exclude = fast list) (unified sampling:
+ *                  the two lists then partition the N samples)
+ *   high-loss samples to the SLOW group (the table's other row):
+ *     slow list  = lsgd_fast_allocation(k_high = floor(lambda N_S), n_fill = N_S - k_high)
+ *     fast list  = lsgd_draw_uniform(n_draw = N_F), with or without the slow list excluded
+ *   unbiased baseline: lsgd_draw_uniform for both groups.
+ * Each list is then cut into per-worker shares with lsgd_worker_share.
+ */
 
 /*
  * lsgd_allocation_sizes — how many of the N samples of an epoch each worker
@@ -179,7 +198,10 @@ LSGD_API lsgd_status lsgd_score_topk(const void* logits, lsgd_dtype dtype, const
  * round and P_S slow workers doing tau_S,
  *     N_F = floor(N * tau_F P_F / (tau_F P_F + tau_S P_S)),   N_S = N - N_F,
  *     k   = floor(lambda * N_F)      (the high-loss part of the fast allocation),
- * N_F in exact integer arithmetic, k in double.  The paper gives the ratios
+ * N_F in exact integer arithmetic; k from the product lambda * N_F in double,
+ * where a product within 2^-51 (relative) below an integer counts as that
+ * integer, so that a decimal lambda gives the decimal result (0.29 * 100 is
+ * 28.999999999999996 in double; k = 29).  The paper gives the ratios
  * only; rounding N_F down and giving the slow workers the rest keeps one epoch
  * at N samples.  Host only.  tau and P values >= 0 with tau_F P_F + tau_S P_S > 0
  * and 0 <= lambda <= 1, else LSGD_ERR_INVALID_ARG.
@@ -190,7 +212,7 @@ LSGD_API lsgd_status lsgd_allocation_sizes(int64_t N, int32_t tau_fast, int32_t 
                                            int64_t* k_high);
 
 /*
- * lsgd_worker_share — "evenly distribute" a list of n sample indices over the
+ * lsgd_worker_share — the even split of a list of n sample indices over the
  * P workers of a group (Section 4.2; Algorithm 1): worker p gets the contiguous
  * entries [begin, end) = [floor(p n / P), floor((p + 1) n / P)).  Shares differ
  * by at most one entry and cover the list exactly once.  Host only.
@@ -200,10 +222,10 @@ LSGD_API lsgd_status lsgd_worker_share(int64_t n, int32_t P, int32_t p, int64_t*
 /*
  * lsgd_draw_uniform — n_draw samples drawn uniformly at random, without
  * replacement, from the samples 0..N-1 that are not listed in exclude_idx
- * (Section 4.2: the slow workers' N_S samples "randomly sampled from the total
- * N samples without replacement"; with an exclusion list, a draw "from the rest
- * of data", e.g. the unified-sampling variant of the appendix where the slow
- * workers draw from what the fast workers left).
+ * (Section 4.2, "Data Allocation for Slow Workers": the slow group's N_S samples
+ * are such a draw from all N samples; with an exclusion list it is a draw from
+ * the remaining samples, e.g. the unified-sampling variant of the appendix in
+ * which the slow workers draw from what the fast workers left).
  *
  * Every sample i gets the random priority q_i = top 30 bits of word (i mod 4)
  * of the Philox4x32-10 block with counter (i div 4, 0, stream_lo, stream_hi) and
@@ -213,7 +235,7 @@ LSGD_API lsgd_status lsgd_worker_share(int64_t n, int32_t P, int32_t p, int64_t*
  * among 30-bit priorities).  The same (N, seed, stream, exclusion) always gives
  * the same result; different `stream` values give independent draws, so a
  * caller can use e.g. stream = 2 * epoch for the fast group and 2 * epoch + 1
- * for the slow group ("separated sampling").
+ * for the slow group (the paper's separated sampling).
  *
  *   exclude_idx  device, [n_exclude] int32 or NULL: distinct indices in [0, N)
  *                (entries outside that range are ignored).
@@ -228,9 +250,9 @@ LSGD_API lsgd_status lsgd_draw_uniform(int64_t N, int64_t n_draw, uint64_t seed,
 
 /*
  * lsgd_fast_allocation — the fast workers' samples for one epoch (Section 4.2,
- * "Data Allocation for Fast Workers"; Algorithm 1: "select ... high-loss
- * samples", then "fill the remainder ... by randomly sampling from the
- * unselected samples"):
+ * "Data Allocation for Fast Workers"; Algorithm 1: the highest-loss samples
+ * first, then the rest of the allocation drawn at random from the samples that
+ * were not selected):
  *     out_idx[0 .. k_high)               the k_high highest-loss samples, as
  *                                        lsgd_topk_select gives them in
  *                                        LSGD_ORDER_LOSS_DESC;
@@ -272,11 +294,11 @@ LSGD_API lsgd_status lsgd_aggregate(const float* const* replicas, const float* w
 /*
  * lsgd_aggregate_round — the aggregation step as one round of the training loop
  * needs it (Eq. 3; the local-SGD update rule of Section 2; Algorithm 1: after
- * "Aggregate the local models" every worker continues from x_{t+1}):
+ * the aggregation step every worker continues from x_{t+1}):
  *
  *   base == NULL:  x_{t+1}[j] = sum_i w_i x_i[j]                         (Eq. 3)
  *   base != NULL:  x_{t+1}[j] = base[j] + sum_i w_i (x_i[j] - base[j])   (Eq. 3 written around base = x_t, the
- *                  form of Section 2's rule "x_t minus the averaged local progress"; identical to Eq. 3 when the
+ *                  form of Section 2's rule, the previous model minus the averaged local progress; identical to Eq. 3 when the
  *                  weights sum to one, and more accurate in fp32 because the differences are small)
  *
  * accumulated in fp32 in ascending i (differences first, one multiply, fused multiply-adds, the base added last).

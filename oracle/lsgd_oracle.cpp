@@ -21,7 +21,7 @@
 // +-0 and all-ignored samples is a convention of this library, not of the
 // paper: parity unpinned for those cases (convention only).  The same holds for
 // which random stream feeds a draw (counter layout, 30-bit priorities, ties by
-// lower index): the paper only says "randomly"; the distribution is pinned, the
+// lower index): the paper asks only for a random draw; the distribution is pinned, the
 // particular bits are this library's convention.
 #include <algorithm>
 #include <cmath>
@@ -59,7 +59,7 @@ inline bool ranks_before(float a, float b) {  // true if a is strictly "higher l
 
 extern "C" {
 
-// Per-sample loss record (Algorithm 1, "record all individual loss"): softmax
+// Per-sample loss record (Algorithm 1, the step that stores every processed sample's loss): softmax
 // cross-entropy with natural log per token, mean over the tokens that are not
 // ignored.
 //   token:   l = (m - x_y) + log(sum_j exp(x_j - m)),  m = max_j x_j
@@ -203,8 +203,10 @@ int oracle_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out
 // Section 4.2: of N samples per epoch the fast workers get
 //   N_F = tau_F P_F / (tau_F P_F + tau_S P_S) * N   (rounded down),
 // the slow workers the rest, N_S = N - N_F (so that one epoch covers N samples),
-// and k = lambda * N_F (rounded down, evaluated in double) of the fast workers'
-// samples are the highest-loss ones.
+// and k = lambda * N_F (rounded down) of the fast workers' samples are the
+// highest-loss ones.  lambda arrives as the double nearest to a decimal fraction,
+// which may lie just below it (0.29 * 100 is 28.999999999999996 in double), so a
+// product within 2^-51 (relative) of an integer counts as that integer.
 int oracle_allocation_sizes(int64_t N, int32_t tau_f, int32_t p_f, int32_t tau_s, int32_t p_s, double lambda,
                             int64_t* n_fast, int64_t* n_slow, int64_t* k_high) {
     if (N < 0 || tau_f < 0 || p_f < 0 || tau_s < 0 || p_s < 0 || !(lambda >= 0.0 && lambda <= 1.0)) return 1;
@@ -213,12 +215,14 @@ int oracle_allocation_sizes(int64_t N, int32_t tau_f, int32_t p_f, int32_t tau_s
     const int64_t nf = static_cast<int64_t>(a * N / (a + b));
     *n_fast = nf;
     *n_slow = N - nf;
-    int64_t k = static_cast<int64_t>(std::floor(lambda * static_cast<double>(nf)));
+    const double prod = lambda * static_cast<double>(nf), near = std::round(prod);
+    int64_t k = std::fabs(prod - near) <= near * 0x1p-51 ? static_cast<int64_t>(near)
+                                                         : static_cast<int64_t>(std::floor(prod));
     *k_high = std::min(std::max<int64_t>(k, 0), nf);
     return 0;
 }
 
-// "Evenly distribute" a list of n entries over P workers: worker p gets the
+// The even split of a list of n entries over P workers: worker p gets the
 // contiguous range [floor(p n / P), floor((p+1) n / P)), so shares differ by at
 // most one entry and together cover the list once.
 int oracle_worker_share(int64_t n, int32_t P, int32_t p, int64_t* begin, int64_t* end) {
@@ -228,9 +232,9 @@ int oracle_worker_share(int64_t n, int32_t P, int32_t p, int64_t* begin, int64_t
     return 0;
 }
 
-// Uniform sampling without replacement (Section 4.2: "randomly selected from the
-// rest of data", "randomly sampled from the total N samples without
-// replacement"): every sample gets an independent random priority; the draw is
+// Uniform sampling without replacement (Section 4.2: the fast group's fill from
+// the samples that were not selected, and the slow group's draw from all N
+// samples): every sample gets an independent random priority; the draw is
 // the m candidates with the highest priority (ties: lower index), listed in that
 // order.  Candidates are the indices 0..N-1 that are not in exclude_idx.
 // Independent, identically distributed priorities make every m-subset of the
@@ -257,9 +261,8 @@ int oracle_priorities(int64_t N, uint64_t seed, uint64_t stream, uint32_t* out) 
     return 0;
 }
 
-// Data allocation for the fast workers (Section 4.2; Algorithm 1, "select ...
-// high-loss samples" then "fill the remainder ... by randomly sampling from the
-// unselected samples"): the k highest-loss samples in loss-descending order,
+// Data allocation for the fast workers (Section 4.2; Algorithm 1, the selection
+// step and the random fill that follows it): the k highest-loss samples in loss-descending order,
 // followed by n_fill samples drawn uniformly without replacement from the other
 // N - k.
 int oracle_fast_allocation(const float* losses, int64_t N, int64_t k, int64_t n_fill, uint64_t seed, uint64_t stream,

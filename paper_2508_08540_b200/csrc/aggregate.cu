@@ -31,9 +31,10 @@ __device__ __forceinline__ float4 mul4(float w, float4 v) { return make_float4(w
 
 // PCT > 0: P known at compile time (all loads of a slice in flight at once).
 // PCT == 0: any P, replicas taken kAggBatch at a time.
+// `out` carries no no-alias promise: it may be one of the replicas (in-place update).
 template <int PCT>
 __global__ void __launch_bounds__(kAggThreads) aggregate_vec4_kernel(const __grid_constant__ AggArgs a, int P,
-                                                                      int64_t n4, float* __restrict__ out) {
+                                                                      int64_t n4, float* out) {
     const int64_t stride = static_cast<int64_t>(gridDim.x) * kAggThreads;
     for (int64_t i = static_cast<int64_t>(blockIdx.x) * kAggThreads + threadIdx.x; i < n4; i += stride) {
         float4 acc;
@@ -64,7 +65,7 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_vec4_kernel(const __gri
 // whole vector when some pointer is not 16-byte aligned.
 __global__ void __launch_bounds__(kAggThreads) aggregate_scalar_kernel(const __grid_constant__ AggArgs a, int P,
                                                                         int64_t begin, int64_t D,
-                                                                        float* __restrict__ out) {
+                                                                        float* out) {
     const int64_t stride = static_cast<int64_t>(gridDim.x) * kAggThreads;
     for (int64_t j = begin + static_cast<int64_t>(blockIdx.x) * kAggThreads + threadIdx.x; j < D; j += stride) {
         float acc = a.w[0] * __ldcs(a.x[0] + j);

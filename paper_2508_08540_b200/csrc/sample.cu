@@ -129,7 +129,12 @@ lsgd_status lsgd_allocation_sizes(int64_t N, int32_t tau_fast, int32_t p_fast, i
     const unsigned __int128 b = static_cast<unsigned __int128>(tau_slow) * static_cast<uint32_t>(p_slow);
     if (a + b == 0) return LSGD_ERR_INVALID_ARG;
     const int64_t nf = static_cast<int64_t>(a * static_cast<unsigned __int128>(N) / (a + b));
-    const int64_t k = static_cast<int64_t>(std::floor(lambda * static_cast<double>(nf)));
+    // floor(lambda N_F); a product that misses the next integer by no more than the rounding of a decimal lambda
+    // and of the multiplication (2^-51 relative) is that integer: 0.29 * 100 = 28.999999999999996 gives 29
+    const double prod = lambda * static_cast<double>(nf);
+    double kf = std::floor(prod);
+    if ((kf + 1.0) - prod <= (kf + 1.0) * 0x1p-51) kf += 1.0;
+    const int64_t k = static_cast<int64_t>(kf);
     *n_fast = nf;
     *n_slow = N - nf;
     *k_high = std::min(std::max<int64_t>(k, 0), nf);

@@ -1,6 +1,6 @@
-// Per-sample loss record (Algorithm 1: "record all individual loss of processed
-// data"): softmax cross-entropy per row of the candidate pool, mean over the
-// unmasked tokens of a sample.
+// Per-sample loss record (Algorithm 1: the step that stores the loss of every
+// processed sample): softmax cross-entropy per row of the candidate pool, mean
+// over the unmasked tokens of a sample.
 //
 // Every row is evaluated from the sum over the OTHER classes (the true class y is left out):
 //     M = max_{j != y} x_j,   S = sum_{j != y} exp(x_j - M)

@@ -112,6 +112,12 @@ def test_allocation_sizes_and_shares_host_only(L):
     nf, ns, k = L.allocation_sizes(1_281_167, 16, 4, 4, 4, 0.3)
     assert nf + ns == 1_281_167 and nf == 1_281_167 * 64 // 80 and k == int(0.3 * nf)
     assert L.allocation_sizes(1000, 5, 0, 2, 3, 0.5) == (0, 1000, 0)
+    # decimal lambdas give the decimal product rounded down (0.29 * 100 is 28.999999999999996 in double)
+    from fractions import Fraction
+
+    for n in (100, 49_612, 1_281_167, 2_000_000_000):
+        for lam in [f"{i / 100:.2f}" for i in range(101)] + ["0.333", "0.0007"]:
+            assert L.allocation_sizes(n, 1, 1, 0, 1, float(lam))[2] == (Fraction(lam) * n).__floor__(), (n, lam)
     for bad in [(-1, 1, 1, 1, 1, 0.5), (10, 0, 0, 0, 0, 0.5), (10, 1, 1, 1, 1, 1.5), (10, 1, 1, 1, 1, float("nan")),
                 (10, -1, 1, 1, 1, 0.5)]:
         with pytest.raises(L.LsgdError) as e:
@@ -190,3 +196,20 @@ def test_binding_fails_loudly_without_the_library(tmp_path):
     ) % (ROOT, str(tmp_path / "liblsgd.so"))
     out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=300)
     assert out.stdout.strip() == "raised True", out.stdout + out.stderr
+
+
+def test_library_sources_never_allocate_device_memory():
+    """The library's contract: the caller owns every buffer.  No source of liblsgd may name an allocating or freeing
+    runtime call (the GPU tests can only watch torch's allocator and the driver's free-memory count)."""
+    import glob
+
+    banned = re.compile(r"\b(cudaMalloc\w*|cudaFree\w*|cudaMemPool\w*|cudaHostAlloc|cudaHostRegister|cuMemAlloc\w*|"
+                        r"cuMemCreate|cuMemMap|cuMemFree\w*)\s*\(")
+    files = sorted(glob.glob(os.path.join(ROOT, "paper_2508_08540_b200", "csrc", "*.cu*")))
+    assert len(files) >= 8
+    for path in files:
+        text = open(path).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        text = re.sub(r"//[^\n]*", "", text)
+        hit = banned.search(text)
+        assert hit is None, f"{os.path.basename(path)} calls {hit.group(1)}"

@@ -92,3 +92,32 @@ def test_epoch_allocation_end_to_end(L, oracle):
     sel = fast.cpu().numpy()[:k]
     rest = np.setdiff1d(np.arange(cfg.N), sel)
     assert lh[sel].min() >= lh[rest].max()
+
+
+@pytest.mark.parametrize("cfg_id,lam", [(1, 1.0), (2, 0.5)])
+def test_high_loss_to_slow_workers_variant(L, oracle, cfg_id, lam):
+    """The appendix's other data allocation (table of data sampling methods, row "High-loss -> CPU"): the SLOW
+    group takes the highest-loss samples, the fast group draws at random; with separated sampling the fast draw is
+    independent, with unified sampling it comes from what the slow group left.  The library has no mode switch:
+    the variant is the same three calls with the groups' sizes exchanged, and every list must match the oracle."""
+    cfg = wl.scaled(wl.CONFIGS[cfg_id], N=20_011)
+    x, y = wl.pool_rows(cfg)
+    nf, ns, _ = L.allocation_sizes(cfg.N, 32, 8, 1, 2, lam)
+    assert (nf, ns) == oracle.allocation_sizes(cfg.N, 32, 8, 1, 2, lam)[:2] and nf + ns == cfg.N
+    k_slow = int(lam * ns)  # the high-loss part of the SLOW allocation
+    losses = L.score_losses(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda())
+    lh = losses.cpu().numpy()
+    slow = L.fast_allocation(losses, k_slow, ns - k_slow, 99, 2)          # top-k_slow, then the random fill
+    fast_separated = L.draw_uniform(cfg.N, nf, 99, 3, device="cuda")      # independent of the slow list
+    fast_unified = L.draw_uniform(cfg.N, nf, 99, 3, exclude_idx=slow)     # from what the slow group left
+    np.testing.assert_array_equal(slow.cpu().numpy(), oracle.fast_allocation(lh, k_slow, ns - k_slow, 99, 2))
+    np.testing.assert_array_equal(fast_separated.cpu().numpy(), oracle.draw_uniform(cfg.N, nf, 99, 3))
+    np.testing.assert_array_equal(fast_unified.cpu().numpy(), oracle.draw_uniform(cfg.N, nf, 99, 3, slow.cpu().numpy()))
+    # the slow group's first k_slow samples are the hardest of the pool (the library's own losses, ties by index)
+    np.testing.assert_array_equal(slow.cpu().numpy()[:k_slow], oracle.topk(lh, k_slow, oracle.LOSS_DESC)[0])
+    # unified: the two groups partition the epoch; separated: the fast draw may overlap the slow list
+    assert np.array_equal(np.sort(np.concatenate([slow.cpu().numpy(), fast_unified.cpu().numpy()])), np.arange(cfg.N))
+    assert np.unique(fast_separated.cpu().numpy()).size == nf
+    # split over the 2 slow and the 8 fast workers
+    assert [L.worker_share(ns, 2, p) for p in range(2)] == [oracle.worker_share(ns, 2, p) for p in range(2)]
+    assert [L.worker_share(nf, 8, p) for p in range(8)] == [oracle.worker_share(nf, 8, p) for p in range(8)]

@@ -154,3 +154,17 @@ def test_fast_allocation_structure(oracle):
     # lambda = 1 (no fill) is the plain top-k; lambda -> 0 (no top-k) is a plain draw
     assert np.array_equal(oracle.fast_allocation(losses, k, 0, 3, 9), order[:k])
     assert np.array_equal(oracle.fast_allocation(losses, 0, fill, 3, 9), oracle.draw_uniform(N, fill, 3, 9))
+
+
+def test_allocation_k_is_the_decimal_product_rounded_down(oracle):
+    """k = floor(lambda N_F) of Section 4.2 for lambda given as a decimal fraction, checked in exact rational
+    arithmetic: the double nearest to a decimal lambda may lie below it (0.29 * 100 = 28.999999999999996)."""
+    from fractions import Fraction
+
+    sizes = [100, 1000, 49_612, 50_000, 1_281_167, 999_983, 2_000_000_000]
+    lams = [f"{i / 100:.2f}" for i in range(0, 101)] + [f"{i / 1000:.3f}" for i in range(1, 1000, 7)] + ["0.3333", "0.0001"]
+    for n in sizes:
+        for lam in lams:
+            nf, ns, k = oracle.allocation_sizes(n, 1, 1, 0, 1, float(lam))  # all samples to the fast group: N_F = n
+            assert nf == n and ns == 0
+            assert k == (Fraction(lam) * n).__floor__(), (n, lam, k)
