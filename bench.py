@@ -483,10 +483,7 @@ def run_gpu(args, cfg):
 def launches_per_step(cfg) -> int:
     """Kernels of liblsgd launched by one step (memsets excluded), from the launch logic of the library."""
     n = 1 + (1 if cfg.T > 1 else 0)                # scorer (+ sequence mean)
-    if cfg.N <= 1024:
-        n += 1                                      # single-CTA selector
-    else:
-        n += 2 + 1 + 1 + 4                          # two more histogram passes, count, emit, four sort passes
+    n += 1                                          # the selector is one kernel at every pool size
     n += 1 + (1 if cfg.D % 4 else 0)                # aggregation (+ ragged tail)
     return n
 

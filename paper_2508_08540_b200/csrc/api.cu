@@ -1,6 +1,7 @@
 // The C ABI of liblsgd (include/lsgd.h): argument checks on the host, then
 // stream-ordered launches.  No device memory is allocated here.
 #include <atomic>
+#include <cstdlib>
 #include <cstring>
 
 #include "lsgd_internal.cuh"
@@ -18,6 +19,16 @@ int sm_count() {
         c.store(v, std::memory_order_relaxed);
     }
     return v;
+}
+
+TestGeometry test_geometry() {
+    TestGeometry g{2147483647, false};
+    if (const char* v = std::getenv("LSGD_TEST_MAX_CTAS")) {
+        const long n = std::strtol(v, nullptr, 10);
+        if (n > 0 && n < 2147483647) g.max_ctas = static_cast<int>(n);
+    }
+    if (const char* v = std::getenv("LSGD_TEST_NO_CLUSTER")) g.no_cluster = v[0] == '1';
+    return g;
 }
 
 size_t score_workspace_bytes(int64_t N, int64_t T, int64_t C) {

@@ -14,16 +14,12 @@ namespace lsgd {
 // Zeroed (together with the selector's histograms) by one memset per call.
 // ---------------------------------------------------------------------------
 struct StatusBlock {
-    int32_t bad_labels;   // tokens with a label outside [0, C) that is not ignore_index
-    int32_t timeout;      // reserved: set by a kernel whose bounded wait ran out (no kernel of this version waits)
+    int32_t bad_labels;      // tokens with a label outside [0, C) that is not ignore_index
+    int32_t timeout;         // set by a block of the selection kernel whose bounded barrier wait ran out
+    uint32_t grid_arrivals;  // the selection kernel's barrier: blocks that have arrived so far, over all its barriers
     uint32_t reserved0;
-    // Radix select: CTAs that finished histogram pass p take a ticket; the last one resolves digit p of the
-    // threshold key once for everybody: the key prefix with digits 0..p placed, and the rank left inside it.
-    uint32_t sel_done[3];
-    uint32_t sel_prefix[3];
-    uint32_t sel_want[3];
-    unsigned long long stream_ticket;  // dynamic row scheduler of the medium-row scorer (offset 48)
-    uint32_t pad[50];
+    unsigned long long stream_ticket;  // dynamic row scheduler of the medium-row scorer
+    uint32_t pad[58];
 };
 static_assert(sizeof(StatusBlock) == 256, "status block is 256 bytes");
 
@@ -36,18 +32,33 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 // ---------------------------------------------------------------------------
 constexpr int kSelPasses = 3;
 constexpr int kSelBins = 2048;            // 11-bit digits (the last digit uses 1024 of them)
-constexpr int kTile = 4096;               // elements per CTA in the count / emit / sort kernels
+constexpr int kTile = 4096;               // smallest selection tile (the per-tile counts are sized for it)
 constexpr int kSmallN = 1024;             // pools up to this size are sorted by one CTA, one entry per thread
-constexpr int kSortBins = 256;            // 8-bit digits of the stable LSD sort of the selected pairs
+constexpr int kSortBits = 9;              // digits of the stable LSD sort of the selected pairs
+constexpr int kSortBins = 1 << kSortBits;
+constexpr int kSortPasses = 4;            // at most: 4 x 9 bits cover a 32-bit key range
+constexpr int kSortMaxRounds = 8;         // a sort tile holds 1024 R entries, R in {1, 2, 4, 8}
+constexpr int kSortDirectTiles = 64;      // the launcher grows R before it uses more sort tiles than this
+constexpr int kMaxClusterBlocks = 8;      // portable cluster size: pools of up to 8 x 8,192 entries run as one cluster
 
 struct TopkWorkspace {       // device pointers carved out of the caller's workspace
     StatusBlock* status;
     uint32_t* hist;          // [kSelPasses][kSelBins]
-    uint32_t* tile_counts;   // [tiles(N)][2]  (#keys above the threshold, #keys equal to it)
+    uint32_t* tile_counts;   // [tiles(N)][4]  (#keys above the threshold, #keys equal to it, largest key, unused)
     uint32_t* keys[2];       // [k] ping-pong: keys of the selected entries
     int32_t* idx[2];         // [k] ping-pong: their indices
-    uint32_t* tile_hist;     // [tiles(k)][kSortBins] digit counts per tile of the current sort pass
+    uint32_t* tile_hist;     // [kSortPasses][sort tiles][kSortBins] digit counts per sort tile and pass
+    uint32_t pass_stride;    // words between the digit counts of consecutive passes
 };
+
+// Test hooks (environment, read at every launch): they change launch geometry only, never results.
+//   LSGD_TEST_MAX_CTAS=n     no kernel of the scorer or the selector uses more than n thread blocks
+//   LSGD_TEST_NO_CLUSTER=1   the selector never runs as a single cluster
+struct TestGeometry {
+    int max_ctas;      // INT_MAX when unset
+    bool no_cluster;
+};
+TestGeometry test_geometry();
 
 struct ScoreWorkspace {
     StatusBlock* status;

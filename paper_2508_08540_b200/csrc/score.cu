@@ -772,10 +772,11 @@ template <typename T>
 cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, int64_t C, int64_t ignore_index,
                         float* row_loss, StatusBlock* status, uint32_t* hist0, cudaStream_t s) {
     const int sms = sm_count();
+    const int64_t max_ctas = test_geometry().max_ctas;
     const int64_t row_bytes = C * static_cast<int64_t>(sizeof(T));
     if (C <= kTinyMaxC) {
         const int64_t tiles = (rows + kTinyThreads - 1) / kTinyThreads;
-        const int grid = static_cast<int>(std::min<int64_t>(tiles, static_cast<int64_t>(sms) * 8));
+        const int grid = static_cast<int>(std::min({tiles, static_cast<int64_t>(sms) * 8, max_ctas}));
         score_tiny_rows_kernel<T><<<grid, kTinyThreads, 0, s>>>(logits, labels, rows, static_cast<int>(C),
                                                                  ignore_index, row_loss, status, hist0);
         return cudaGetLastError();
@@ -795,7 +796,7 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
             err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynSmem));
             if (err != cudaSuccess) return;
             const int64_t tiles = (rows + tile_rows - 1) / tile_rows;
-            const int grid = static_cast<int>(std::min<int64_t>(tiles, static_cast<int64_t>(sms) * blocks_per_sm(kernel, kGroupThreads, smem)));
+            const int grid = static_cast<int>(std::min({tiles, static_cast<int64_t>(sms) * blocks_per_sm(kernel, kGroupThreads, smem), max_ctas}));
             kernel<<<grid, kGroupThreads, smem, s>>>(logits, labels, rows, static_cast<int>(C), ignore_index, row_loss,
                                                      status, hist0, stage_bytes);
             err = cudaGetLastError();
@@ -804,8 +805,9 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
             constexpr int LN = decltype(lanes_tag)::value;
             if (cb == 16) go(score_group_rows_kernel<T, LN, 16>, LN);
             else if (cb == 8) go(score_group_rows_kernel<T, LN, 8>, LN);
-            else if (cb == 4 && sizeof(T) == 2) go(score_group_rows_kernel<T, LN, 4>, LN);
-            else go(score_group_rows_kernel<T, LN, 0>, LN);  // (4-byte chunks of fp32 are single elements)
+            else if (cb == 4 && sizeof(T) == 2) {
+                if constexpr (sizeof(T) == 2) go(score_group_rows_kernel<T, LN, 4>, LN);  // (4-byte chunks of fp32 are single elements)
+            } else go(score_group_rows_kernel<T, LN, 0>, LN);
         };
         // rows per tile (256 / L) times bytes per row: at most 32 KB per stage (64 x 512, 32 x 1024, 16 x 2048), plus padding
         if (row_bytes <= 512) by_chunk(std::integral_constant<int, 4>{});
@@ -815,8 +817,8 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
     }
     if (row_bytes <= kStreamMaxRowBytes) {
         const int64_t want = (rows + kStreamThreads / 32 - 1) / (kStreamThreads / 32);
-        const int grid = static_cast<int>(std::min<int64_t>(
-            want, static_cast<int64_t>(sms) * blocks_per_sm(score_stream_rows_kernel<T>, kStreamThreads, 0)));
+        const int grid = static_cast<int>(std::min({
+            want, static_cast<int64_t>(sms) * blocks_per_sm(score_stream_rows_kernel<T>, kStreamThreads, 0), max_ctas}));
         // rows per ticket: about 32 KB of logits
         const int batch = static_cast<int>(std::max<int64_t>(1, 32768 / row_bytes));
         score_stream_rows_kernel<T><<<grid, kStreamThreads, 0, s>>>(logits, labels, rows, static_cast<int>(C),
@@ -824,7 +826,7 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
         return cudaGetLastError();
     }
     // longer rows are few per byte: a warp per row would leave most of the machine idle, so a CTA takes each
-    const int grid = static_cast<int>(std::min<int64_t>(rows, static_cast<int64_t>(sms) * 8));
+    const int grid = static_cast<int>(std::min({rows, static_cast<int64_t>(sms) * 8, max_ctas}));
     score_huge_rows_kernel<T><<<grid, kCtaThreads, 0, s>>>(logits, labels, rows, C, ignore_index, row_loss, status,
                                                             hist0);
     return cudaGetLastError();
@@ -844,7 +846,7 @@ cudaError_t launch_score(const void* logits, lsgd_dtype dt, const int64_t* label
                         : launch_rows(static_cast<const __nv_bfloat16*>(logits), labels, rows, C, ignore_index,
                                       row_loss, ws.status, row_hist, s);
     if (e != cudaSuccess || T == 1) return e;
-    const int grid = static_cast<int>(std::min<int64_t>((N + 7) / 8, static_cast<int64_t>(sm_count()) * 8));
+    const int grid = static_cast<int>(std::min({(N + 7) / 8, static_cast<int64_t>(sm_count()) * 8, static_cast<int64_t>(test_geometry().max_ctas)}));
     seq_mean_kernel<<<grid, 256, 0, s>>>(ws.token_loss, labels, N, T, ignore_index, losses, hist0);
     return cudaGetLastError();
 }

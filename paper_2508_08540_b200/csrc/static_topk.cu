@@ -20,12 +20,12 @@ namespace {
 // that it is a compile-time constant (checked against the run-time formula below).
 constexpr size_t kMaxN = LSGD_STATIC_TOPK_MAX_N;
 constexpr size_t kMaxTiles = (kMaxN + kTile - 1) / kTile;
-constexpr size_t kMaxSortTiles = 128;  // the sort's digit counts: up to 131,072 entries in tiles of 1024, more in tiles of 4096
-static_assert(kMaxSortTiles >= kMaxTiles, "the sort's tile bound covers the largest pool");
+constexpr size_t kMaxSortTiles = kSortDirectTiles;  // pools of this size never use more sort tiles
+static_assert(kMaxN <= size_t{kSortDirectTiles} * 1024 * kSortMaxRounds, "the sort's tile bound covers the largest pool");
 constexpr size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 constexpr size_t kScratchBytes = sizeof(StatusBlock) + up256(sizeof(uint32_t) * kSelPasses * kSelBins) +
-                                 up256(sizeof(uint32_t) * 4 * kMaxSortTiles * kSortBins) +
-                                 up256(sizeof(uint32_t) * 2 * kMaxTiles) + 4 * up256(sizeof(uint32_t) * kMaxN);
+                                 up256(sizeof(uint32_t) * kSortPasses * kMaxSortTiles * kSortBins) +
+                                 up256(sizeof(uint32_t) * 4 * kMaxTiles) + 4 * up256(sizeof(uint32_t) * kMaxN);
 
 // The scratch itself.  In host code this name is only a handle for the runtime's
 // symbol table, never an address a kernel may be given: the device address is

@@ -5,48 +5,59 @@
 // order-preserving 32-bit keys (loss_key), so everything below is integer work
 // and the result is exact and bit-reproducible.
 //
-//   1. radix select: three histogram passes (11 + 11 + 10 bits, most significant
-//      digit first) find the key T of the k-th entry and r, the number of entries
-//      equal to T that still belong to the selection;
-//   2. ordered compaction: per-tile counts, then an emit pass that keeps every
-//      key > T and the r lowest-index keys == T, writing them in index order
-//      (scan-based positions: no atomics decide an order);
-//   3. for loss-descending output, a stable LSD radix sort (four 8-bit digits) of
-//      the k (key, index) pairs; stability turns the index-ascending input order
-//      into the required tie-break.  Each scatter pass accumulates the digit
-//      counts of the next pass, so the sort is one kernel per digit.
-// Pools of at most kSmallN entries are sorted whole by a single CTA instead.
-//
-// The kernels are short and depend on one another, so their latency is what
-// counts: each digit of the threshold is resolved once, by the last CTA to
-// finish its histogram pass (a ticket, no waiting), and every kernel is launched
-// so that it can be scheduled while its predecessor drains (it waits for the
-// predecessor's completion before its first global access).
+// One kernel does the whole selection, in phases separated by a barrier over all
+// its thread blocks:
+//   1. radix select: three digit histograms (11 + 11 + 10 bits, most significant
+//      first; the first one may come ready-made from the scorer) find the key T of
+//      the k-th entry and r, the number of entries equal to T that still belong to
+//      the selection.  Every block resolves a digit for itself from the finished
+//      histogram; a block keeps the keys of its first tile in registers throughout;
+//   2. per-tile counts of keys above / equal to T (and the largest key);
+//   3. ordered compaction: every key > T and the r lowest-index keys == T are
+//      written in index order (scan-based positions: no atomics decide an order);
+//   4. for loss-descending output, a stable LSD radix sort of the k (key, index)
+//      pairs on u = (largest key - key) in 9-bit digits: only as many passes as
+//      u's range needs (three for losses that span up to 16 binades above T, none
+//      if all selected keys are equal); stability turns the index-ascending input
+//      order into the required tie-break.  Each scatter counts the next digit per
+//      destination tile, so a pass is one phase.
+// The kernel runs either as ONE thread-block cluster (pools of up to 65,536
+// entries: the barrier is the cluster's hardware barrier) or as a cooperative
+// launch with one block per multiprocessor (all blocks resident by construction;
+// the barrier is an arrival counter in the status block, polled with a limit: if
+// it ever ran out, the block would set the status block's timeout word and
+// return, and the other blocks would follow).
+// Pools of at most kSmallN entries are sorted whole by a single block instead.
 #include <algorithm>
 
 #include "lsgd_internal.cuh"
 
 namespace lsgd {
 
-// The sort of the selected pairs works on tiles of 1024 entries when k is small (more, shorter CTAs: the pass is
-// latency-bound) and of kTile entries otherwise (fewer tiles to prefix over).
-constexpr int64_t kSmallSortK = 131072;
-static int sort_tile_shift(int64_t k) { return k <= kSmallSortK ? 10 : 12; }
-static size_t sort_tiles(int64_t k) { return static_cast<size_t>((k + (int64_t{1} << sort_tile_shift(k)) - 1) >> sort_tile_shift(k)); }
-// Tiles reserved for the digit counts: an upper bound of sort_tiles() that grows with k, so that a workspace sized
-// for k also serves every smaller k.
-static size_t sort_tiles_bound(int64_t k) {
-    const size_t small = static_cast<size_t>((std::min<int64_t>(k, kSmallSortK) + 1023) / 1024);
-    return std::max(small, static_cast<size_t>((k + kTile - 1) / kTile));
+// ---------------------------------------------------------------------------
+// Geometry that the workspace layout depends on (host arithmetic only).
+// ---------------------------------------------------------------------------
+// Entries per sort tile: 1024 R with R in {1, 2, 4, 8}, the smallest that needs at most `max_tiles` tiles.
+static int sort_rounds_for(int64_t k, int64_t max_tiles) {
+    for (int r = 1; r < kSortMaxRounds; r <<= 1)
+        if ((k + 1024 * r - 1) / (1024 * r) <= max_tiles) return r;
+    return kSortMaxRounds;
 }
+// Upper bound of the number of sort tiles for any geometry the launcher may pick; grows with k, so that a
+// workspace sized for k also serves every smaller k.
+static size_t sort_tiles_bound(int64_t k) {
+    if (k <= int64_t{kSortDirectTiles} * 1024 * kSortMaxRounds) return static_cast<size_t>(std::min<int64_t>(kSortDirectTiles, (k + 1023) / 1024));
+    return static_cast<size_t>((k + 1024 * kSortMaxRounds - 1) / (1024 * kSortMaxRounds));
+}
+static size_t sort_count_words(int64_t k) { return static_cast<size_t>(kSortPasses) * sort_tiles_bound(k) * kSortBins; }
 
 size_t topk_workspace_bytes(int64_t N, int64_t k) {
     if (N < 0 || k < 0 || k > N) return 0;
     const size_t tiles_n = static_cast<size_t>((N + kTile - 1) / kTile);
     size_t b = sizeof(StatusBlock);
     b += align_up(sizeof(uint32_t) * kSelPasses * kSelBins);
-    b += align_up(sizeof(uint32_t) * 4 * sort_tiles_bound(k) * kSortBins);
-    b += align_up(sizeof(uint32_t) * 2 * tiles_n);
+    b += align_up(sizeof(uint32_t) * sort_count_words(k));
+    b += align_up(sizeof(uint32_t) * 4 * tiles_n);
     b += 4 * align_up(sizeof(uint32_t) * static_cast<size_t>(k));
     return b;
 }
@@ -54,7 +65,7 @@ size_t topk_workspace_bytes(int64_t N, int64_t k) {
 // Bytes at the start of the workspace that one memset must clear before a call.
 static size_t topk_zero_bytes(int64_t k) {
     return sizeof(StatusBlock) + align_up(sizeof(uint32_t) * kSelPasses * kSelBins) +
-           align_up(sizeof(uint32_t) * 4 * sort_tiles_bound(k) * kSortBins);
+           align_up(sizeof(uint32_t) * sort_count_words(k));
 }
 
 TopkWorkspace carve_topk(void* ws, int64_t N, int64_t k) {
@@ -66,9 +77,10 @@ TopkWorkspace carve_topk(void* ws, int64_t N, int64_t k) {
     w.hist = reinterpret_cast<uint32_t*>(p);
     p += align_up(sizeof(uint32_t) * kSelPasses * kSelBins);
     w.tile_hist = reinterpret_cast<uint32_t*>(p);
-    p += align_up(sizeof(uint32_t) * 4 * sort_tiles_bound(k) * kSortBins);
+    w.pass_stride = static_cast<uint32_t>(sort_tiles_bound(k) * kSortBins);
+    p += align_up(sizeof(uint32_t) * sort_count_words(k));
     w.tile_counts = reinterpret_cast<uint32_t*>(p);
-    p += align_up(sizeof(uint32_t) * 2 * tiles_n);
+    p += align_up(sizeof(uint32_t) * 4 * tiles_n);
     const size_t kb = align_up(sizeof(uint32_t) * static_cast<size_t>(k));
     w.keys[0] = reinterpret_cast<uint32_t*>(p);
     w.keys[1] = reinterpret_cast<uint32_t*>(p + kb);
@@ -83,17 +95,74 @@ cudaError_t zero_topk_workspace(void* ws, int64_t k, cudaStream_t s) {
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kPerThread = kTile / kThreads;  // 16
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+constexpr int kCounterPitch = kSortBins + 1;  // odd pitch: a warp can read one bin of all 32 rows without bank conflicts
+constexpr size_t kDynSmemBytes = sizeof(uint32_t) * kWarps * kCounterPitch;
+constexpr uint32_t kMaxPolls = 1u << 21;      // barrier polls before a block gives up (seconds; never reached when all blocks are resident)
+
+struct SelectParams {
+    const float* losses;
+    int64_t N;
+    uint32_t k;
+    int order;
+    int32_t* out_idx;
+    float* out_vals;
+    TopkWorkspace ws;
+    uint32_t sort_tiles;  // tiles of 1024 * sort_rounds entries over the k selected pairs
+    int sort_rounds;
+    int hist0_ready;      // the first digit's histogram was accumulated by the scorer
+};
 
 __device__ __forceinline__ uint32_t digit_of(uint32_t key, int pass) {
     return pass == 0 ? key >> 21 : pass == 1 ? (key >> 10) & 0x7FFu : key & 0x3FFu;
 }
+__device__ __forceinline__ uint32_t prefix_mask(int pass) { return pass == 0 ? 0u : pass == 1 ? 0xFFE00000u : 0xFFFFFC00u; }
 
-// Block-wide exclusive scan of one value per thread (kThreads threads).
-// `scratch` holds kThreads / 32 + 1 words.  Returns the exclusive prefix; the
-// block total is left in scratch[kThreads / 32].
-__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* scratch) {
+__device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Barrier over all blocks of the kernel, with the other blocks' global writes visible afterwards (read them with
+// __ldcg).  CLUSTER: the grid is one cluster, the barrier is the cluster's.  Otherwise (cooperative launch): an
+// arrival counter that only grows; barrier number e is passed once e * gridDim.x arrivals are in.  Returns false
+// if the wait ran out (or another block's did): the caller returns at once.
+template <bool CLUSTER>
+__device__ __forceinline__ bool grid_sync(StatusBlock* st, uint32_t& epoch) {
+    if constexpr (CLUSTER) {
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        return true;
+    } else {
+        __shared__ int ok_s;
+        ++epoch;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const uint32_t target = epoch * gridDim.x;
+            __threadfence();
+            atomicAdd(&st->grid_arrivals, 1u);
+            int ok = 1;
+            uint32_t polls = 0;
+            while (ld_acquire(&st->grid_arrivals) < target) {
+                if (++polls > kMaxPolls || ((polls & 63u) == 0 && *reinterpret_cast<volatile int32_t*>(&st->timeout) != 0)) {
+                    ok = 0;
+                    break;
+                }
+                __nanosleep(32);
+            }
+            if (!ok) atomicExch(&st->timeout, 1);
+            __threadfence();
+            ok_s = ok;
+        }
+        __syncthreads();
+        return ok_s != 0;
+    }
+}
+
+// Block-wide exclusive scan of one value per thread.  `warp_tot` holds kWarps + 1 words; the block total is left
+// in warp_tot[kWarps].
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* warp_tot) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t inc = v;
 #pragma unroll
@@ -101,49 +170,37 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
         const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
         if (lane >= o) inc += n;
     }
-    __syncthreads();  // scratch may still be read from an earlier call
-    if (lane == 31) scratch[warp] = inc;
+    __syncthreads();  // warp_tot may still be read from an earlier call
+    if (lane == 31) warp_tot[warp] = inc;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        uint32_t run = 0;
-        for (int w = 0; w < kThreads / 32; ++w) {
-            const uint32_t c = scratch[w];
-            scratch[w] = run;
-            run += c;
+    if (warp == 0) {
+        const uint32_t w = warp_tot[lane];
+        uint32_t wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, wi, o);
+            if (lane >= o) wi += n;
         }
-        scratch[kThreads / 32] = run;
+        warp_tot[lane] = wi - w;
+        if (lane == 31) warp_tot[kWarps] = wi;
     }
     __syncthreads();
-    return scratch[warp] + inc - v;
+    return warp_tot[warp] + inc - v;
 }
 
-// Walks a histogram from its highest bin down and finds the bin that holds the
-// `want`-th entry (1-based).  On return (all threads): bin, and `want` reduced by
-// the entries in the bins above it.
-__device__ void find_bin(const uint32_t* hist, int nbins, uint32_t& want, uint32_t& bin, uint32_t* scratch,
-                         uint32_t* result) {
-    const int per = nbins / kThreads;  // 8 or 4
-    // thread t owns bins [nbins - 1 - t*per - (per - 1), nbins - 1 - t*per], highest first
-    uint32_t c[8];
-    uint32_t sum = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i)  // all loads in flight together
-        c[i] = i < per ? __ldcg(hist + (nbins - 1 - (threadIdx.x * per + i))) : 0u;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) sum += c[i];
-    const uint32_t before = block_exclusive_scan(sum, scratch);
-    if (before < want && want <= before + sum) {
-        uint32_t run = before;
-        bool found = false;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            if (!found && i < per && want <= run + c[i]) {
-                result[0] = nbins - 1 - (threadIdx.x * per + i);
-                result[1] = want - run;
-                found = true;
-            }
-            run += c[i];
-        }
+// Walks a finished histogram (global memory) from its highest bin down and finds the bin that holds the `want`-th
+// entry (1-based).  On return (all threads): bin, and `want` reduced by the entries in the bins above it.
+__device__ void find_bin(const uint32_t* hist, int nbins, uint32_t& want, uint32_t& bin, uint32_t* warp_tot, uint32_t* result) {
+    // thread t owns bins nbins - 1 - 2 t and nbins - 2 - 2 t (or the single bin nbins - 1 - t), highest first
+    const bool two = nbins == 2 * kThreads;
+    const int b0 = two ? nbins - 1 - 2 * static_cast<int>(threadIdx.x) : nbins - 1 - static_cast<int>(threadIdx.x);
+    const uint32_t c0 = __ldcg(hist + b0);
+    const uint32_t c1 = two ? __ldcg(hist + b0 - 1) : 0u;
+    const uint32_t before = block_exclusive_scan(c0 + c1, warp_tot);
+    if (before < want && want <= before + c0 + c1) {
+        const bool first = want <= before + c0;
+        result[0] = first ? b0 : b0 - 1;
+        result[1] = first ? want - before : want - before - c0;
     }
     __syncthreads();
     bin = result[0];
@@ -151,52 +208,16 @@ __device__ void find_bin(const uint32_t* hist, int nbins, uint32_t& want, uint32
     __syncthreads();
 }
 
-// After a histogram pass: the last CTA to get here resolves digit `pass` of the threshold from the finished
-// histogram and publishes (prefix, rank left) in the status block.  Every thread of the CTA must call it, after
-// its last atomic on the histogram.  `prefix_in`, `want_in`: the state before this digit.
-__device__ void publish_digit(StatusBlock* status, const uint32_t* hist, int pass, uint32_t prefix_in, uint32_t want_in,
-                              uint32_t* scratch, uint32_t* result) {
-    __shared__ uint32_t last_s;
-    __threadfence();  // this thread's histogram atomics are ordered before the ticket
-    __syncthreads();
-    if (threadIdx.x == 0) last_s = atomicAdd(&status->sel_done[pass], 1u) == gridDim.x - 1;
-    __syncthreads();
-    if (!last_s) return;
-    __threadfence();
-    uint32_t want = want_in, bin;
-    find_bin(hist + pass * kSelBins, pass == 2 ? 1024 : kSelBins, want, bin, scratch, result);
-    if (threadIdx.x == 0) {
-        status->sel_prefix[pass] = prefix_in | (pass == 0 ? bin << 21 : pass == 1 ? bin << 10 : bin);
-        status->sel_want[pass] = want;
-    }
-}
-
-// Resolves the digits of the threshold key that passes [0, upto) fixed.
-// Returns the key prefix (digits placed, lower bits zero) and the rank left
-// inside that prefix.
-__device__ uint32_t resolve_prefix(const uint32_t* hist, int upto, uint32_t k, uint32_t& want, uint32_t* scratch,
-                                   uint32_t* result) {
-    uint32_t prefix = 0;
-    want = k;
-    for (int p = 0; p < upto; ++p) {
-        uint32_t bin;
-        find_bin(hist + p * kSelBins, p == 2 ? 1024 : kSelBins, want, bin, scratch, result);
-        prefix |= p == 0 ? bin << 21 : p == 1 ? bin << 10 : bin;
-    }
-    return prefix;
-}
-
-__device__ __forceinline__ uint32_t prefix_mask(int pass) { return pass == 0 ? 0u : pass == 1 ? 0xFFE00000u : 0xFFFFFC00u; }
-
-// Loads the 16 keys thread `threadIdx.x` owns in tile `tile` (consecutive
-// indices), 0 beyond N.  Key 0 belongs to no loss (loss_key never returns it).
-__device__ __forceinline__ void load_keys(const float* __restrict__ losses, int64_t N, int64_t base, uint32_t (&key)[kPerThread]) {
-    if (base + kPerThread <= N && (reinterpret_cast<uintptr_t>(losses + base) & 15) == 0) {
-        float4 q[kPerThread / 4];
+// Loads the E keys a thread owns (consecutive indices from `base`), 0 beyond N.  Key 0 belongs to no loss
+// (loss_key never returns it) and is below every threshold.
+template <int E>
+__device__ __forceinline__ void load_keys(const float* __restrict__ losses, int64_t N, int64_t base, uint32_t (&key)[E]) {
+    if (base + E <= N && (reinterpret_cast<uintptr_t>(losses + base) & 15) == 0) {
+        float4 q[E / 4];
 #pragma unroll
-        for (int i = 0; i < kPerThread / 4; ++i) q[i] = reinterpret_cast<const float4*>(losses + base)[i];
+        for (int i = 0; i < E / 4; ++i) q[i] = reinterpret_cast<const float4*>(losses + base)[i];
 #pragma unroll
-        for (int i = 0; i < kPerThread / 4; ++i) {
+        for (int i = 0; i < E / 4; ++i) {
             key[4 * i] = loss_key(q[i].x);
             key[4 * i + 1] = loss_key(q[i].y);
             key[4 * i + 2] = loss_key(q[i].z);
@@ -205,177 +226,18 @@ __device__ __forceinline__ void load_keys(const float* __restrict__ losses, int6
         return;
     }
 #pragma unroll
-    for (int i = 0; i < kPerThread; ++i) {
+    for (int i = 0; i < E; ++i) {
         const int64_t j = base + i;
         key[i] = j < N ? loss_key(losses[j]) : 0u;
     }
 }
 
-// Histogram pass `pass`: counts digit `pass` of the keys that match the prefix fixed by the earlier passes, then
-// (last CTA) resolves that digit.  `prev_published`: the state after the previous pass is in the status block;
-// otherwise (pass 1 after a scorer that built the first histogram itself) digit 0 is resolved here by every CTA.
-__global__ void __launch_bounds__(kThreads)
-select_hist_kernel(const float* __restrict__ losses, int64_t N, uint32_t k, int pass, bool prev_published,
-                   uint32_t* hist, StatusBlock* status) {
-    __shared__ uint32_t hist_s[kSelBins];
-    __shared__ uint32_t scratch[kThreads / 32 + 1];
-    __shared__ uint32_t result[2];
-    for (int i = threadIdx.x; i < kSelBins; i += kThreads) hist_s[i] = 0;
-    grid_dependency_wait();
-    uint32_t want = k, prefix = 0;
-    if (pass > 0) {
-        if (prev_published) {
-            prefix = __ldcg(&status->sel_prefix[pass - 1]);
-            want = __ldcg(&status->sel_want[pass - 1]);
-        } else {
-            prefix = resolve_prefix(hist, pass, k, want, scratch, result);
-        }
-    }
-    __syncthreads();
-    const uint32_t mask = prefix_mask(pass);
-    for (int64_t tile = blockIdx.x; tile * kTile < N; tile += gridDim.x) {
-        const int64_t base = tile * kTile;
-        float v[kPerThread];
-#pragma unroll
-        for (int i = 0; i < kPerThread; ++i) {  // all loads first: they are independent
-            const int64_t j = base + i * kThreads + threadIdx.x;
-            v[i] = j < N ? losses[j] : 0.f;
-        }
-#pragma unroll
-        for (int i = 0; i < kPerThread; ++i) {
-            const int64_t j = base + i * kThreads + threadIdx.x;
-            const uint32_t key = loss_key(v[i]);
-            const bool in = j < N && (key & mask) == prefix;
-            if (pass == 0) {
-                // every key counts and losses crowd into a few bins: one atomic per distinct digit and warp
-                const uint32_t d = in ? digit_of(key, 0) : 0xFFFFFFFFu;
-                const uint32_t peers = __match_any_sync(0xFFFFFFFFu, d);
-                if (in && (threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist_s[d], __popc(peers));
-            } else if (in) {
-                atomicAdd(&hist_s[digit_of(key, pass)], 1u);
-            }
-        }
-    }
-    __syncthreads();
-    grid_launch_dependents();  // only the flush and the digit's resolution are left
-    uint32_t* out = hist + pass * kSelBins;
-    for (int i = threadIdx.x; i < kSelBins; i += kThreads)
-        if (hist_s[i]) atomicAdd(&out[i], hist_s[i]);
-    publish_digit(status, hist, pass, prefix, want, scratch, result);
-}
-
-// Per tile: how many keys are above the threshold, how many equal it.
-__global__ void __launch_bounds__(kThreads)
-select_count_kernel(const float* __restrict__ losses, int64_t N, const StatusBlock* status, uint32_t* tile_counts) {
-    __shared__ uint32_t cnt[2];
-    grid_dependency_wait();
-    const uint32_t T = __ldcg(&status->sel_prefix[kSelPasses - 1]);
-    for (int64_t tile = blockIdx.x; tile * kTile < N; tile += gridDim.x) {
-        if (threadIdx.x < 2) cnt[threadIdx.x] = 0;
-        __syncthreads();
-        uint32_t gt = 0, eq = 0;
-        float v[kPerThread];
-#pragma unroll
-        for (int i = 0; i < kPerThread; ++i) {
-            const int64_t j = tile * kTile + i * kThreads + threadIdx.x;
-            v[i] = j < N ? losses[j] : 0.f;
-        }
-#pragma unroll
-        for (int i = 0; i < kPerThread; ++i) {
-            const int64_t j = tile * kTile + i * kThreads + threadIdx.x;
-            const uint32_t key = j < N ? loss_key(v[i]) : 0u;  // key 0 belongs to no loss and is below every threshold
-            gt += key > T;
-            eq += key == T;
-        }
-        gt = warp_sum(static_cast<int>(gt));
-        eq = warp_sum(static_cast<int>(eq));
-        if ((threadIdx.x & 31) == 0) {
-            atomicAdd(&cnt[0], gt);
-            atomicAdd(&cnt[1], eq);
-        }
-        __syncthreads();
-        if (threadIdx.x < 2) tile_counts[2 * tile + threadIdx.x] = cnt[threadIdx.x];
-        __syncthreads();
-        if (tile + gridDim.x >= (N + kTile - 1) / kTile) grid_launch_dependents();  // this CTA's last tile is done
-    }
-}
-
-// Emit: keeps every key above the threshold and the first `r` (by index) equal
-// to it, in index order.  Positions come from the tile counts and an in-tile
-// scan.  DIRECT: write the final index-ascending result; otherwise write the
-// (key, index) pairs for the sort and count their first sort digit.
-template <bool DIRECT>
-__global__ void __launch_bounds__(kThreads)
-select_emit_kernel(const float* __restrict__ losses, int64_t N, const StatusBlock* status,
-                   const uint32_t* tile_counts, int32_t* __restrict__ out_idx,
-                   float* __restrict__ out_vals, uint32_t* __restrict__ out_keys, uint32_t* __restrict__ tile_hist,
-                   int sort_shift) {
-    __shared__ uint32_t scratch[kThreads / 32 + 1];
-    __shared__ uint32_t pre[2];
-    grid_dependency_wait();
-    const uint32_t T = __ldcg(&status->sel_prefix[kSelPasses - 1]);
-    const uint32_t r = __ldcg(&status->sel_want[kSelPasses - 1]);
-    for (int64_t tile = blockIdx.x; tile * kTile < N; tile += gridDim.x) {
-        // entries above / equal to the threshold in the tiles before this one
-        if (threadIdx.x < 2) pre[threadIdx.x] = 0;
-        __syncthreads();
-        uint32_t gt = 0, eq = 0;
-        for (int64_t t = threadIdx.x; t < tile; t += kThreads) {
-            gt += __ldcg(tile_counts + 2 * t);
-            eq += __ldcg(tile_counts + 2 * t + 1);
-        }
-        gt = warp_sum(static_cast<int>(gt));
-        eq = warp_sum(static_cast<int>(eq));
-        if ((threadIdx.x & 31) == 0) {
-            atomicAdd(&pre[0], gt);
-            atomicAdd(&pre[1], eq);
-        }
-        __syncthreads();
-        const uint32_t gt_before = pre[0], eq_before = pre[1];
-
-        const int64_t base = tile * kTile + static_cast<int64_t>(threadIdx.x) * kPerThread;
-        uint32_t key[kPerThread];
-        load_keys(losses, N, base, key);
-        if (tile + gridDim.x >= (N + kTile - 1) / kTile) grid_launch_dependents();  // this CTA's last tile
-        uint32_t my_gt = 0, my_eq = 0;
-#pragma unroll
-        for (int i = 0; i < kPerThread; ++i) {
-            my_gt += key[i] > T;
-            my_eq += (key[i] == T);
-        }
-        // one scan for both counts: each is at most kTile = 4096 < 2^16
-        const uint32_t packed = block_exclusive_scan(my_gt | (my_eq << 16), scratch);
-        uint32_t gt_run = gt_before + (packed & 0xFFFFu);
-        uint32_t eq_run = eq_before + (packed >> 16);
-#pragma unroll
-        for (int i = 0; i < kPerThread; ++i) {
-            const bool above = key[i] > T;
-            const bool tie = key[i] == T;
-            if (above || (tie && eq_run < r)) {
-                const uint32_t pos = gt_run + min(eq_run, r);
-                const int64_t j = base + i;
-                if (DIRECT) {
-                    out_idx[pos] = static_cast<int32_t>(j);
-                    if (out_vals) out_vals[pos] = losses[j];
-                } else {
-                    out_idx[pos] = static_cast<int32_t>(j);
-                    out_keys[pos] = key[i];
-                    atomicAdd(&tile_hist[(pos >> sort_shift) * kSortBins + (255u - (key[i] & 0xFFu))], 1u);
-                }
-            }
-            gt_run += above;
-            eq_run += tie;
-        }
-        __syncthreads();
-    }
-}
-
-// Lanes of the warp whose 8-bit digit equals this lane's, among the lanes with `live` set (0 for a lane that is
-// not live).  Nine votes; cheaper here than the generic match instruction.
-__device__ __forceinline__ uint32_t match_digit8(uint32_t d, bool live) {
+// Lanes of the warp whose 9-bit digit equals this lane's, among the lanes with `live` set (0 for a lane that is
+// not live).  Ten votes; cheaper here than the generic match instruction.
+__device__ __forceinline__ uint32_t match_digit(uint32_t d, bool live) {
     uint32_t peers = __ballot_sync(0xFFFFFFFFu, live);
 #pragma unroll
-    for (int b = 0; b < 8; ++b) {
+    for (int b = 0; b < kSortBits; ++b) {
         const bool bit = (d >> b) & 1u;
         const uint32_t m = __ballot_sync(0xFFFFFFFFu, bit);
         peers &= bit ? m : ~m;
@@ -383,161 +245,324 @@ __device__ __forceinline__ uint32_t match_digit8(uint32_t d, bool live) {
     return live ? peers : 0u;
 }
 
-// One stable LSD pass over the selected pairs, on digit `pass` (8 bits, least
-// significant first), larger digits first.  Reads the digit counts per source
-// tile, ranks the tile's entries stably (warp match + per-warp counters), and
-// scatters.  Unless LAST, also counts the next digit per destination tile.
-// The pass is latency-bound (a short chain of dependent steps per tile), so a
-// tile is spread over 32 warps: four ranking rounds per warp instead of sixteen.
-constexpr int kSortThreads = 1024;
-
-template <bool LAST, int kRounds>  // kRounds rounds of 32 consecutive entries per warp: tiles of 1024 kRounds entries
-__global__ void __launch_bounds__(kSortThreads)
-sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restrict__ idx_in, uint32_t k, int pass,
-                    const uint32_t* __restrict__ tile_hist, uint32_t* __restrict__ keys_out,
-                    int32_t* __restrict__ idx_out, uint32_t* __restrict__ next_hist,
-                    const float* __restrict__ losses, float* __restrict__ out_vals) {
-    constexpr int kWarps = kSortThreads / 32;
-    constexpr uint32_t kSortTile = kSortThreads * kRounds;
-    constexpr int kSortShift = kRounds == 1 ? 10 : 12;
-    static_assert(kRounds == 1 || kRounds == 4, "tiles of 1024 or 4096 entries");
-    static_assert(kSortBins == 256 && kSortThreads >= kSortBins, "one thread per digit in the scans");
-    __shared__ uint32_t counters[kWarps][kSortBins];
-    __shared__ uint32_t base_s[kSortBins];
-    __shared__ uint32_t tot_s[kSortBins];
-    constexpr int kParts = kSortThreads / kSortBins;
-    __shared__ uint32_t part_tot[kParts][kSortBins], part_bef[kParts][kSortBins];
+// E: keys per thread of a selection tile (tiles of 1024 E entries; block b takes tiles b, b + gridDim.x, ...).
+template <int E, bool CLUSTER>
+__global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_constant__ SelectParams p) {
+    extern __shared__ __align__(16) uint32_t dyn_smem[];  // selection: hist_s[kSelBins]; sort: counters[kWarps][kCounterPitch]
+    __shared__ uint32_t warp_tot[kWarps + 1];
+    __shared__ uint32_t result[2];
+    __shared__ uint32_t red[3];
+    __shared__ uint32_t part_tot[2][kSortBins], part_bef[2][kSortBins];
+    __shared__ uint32_t base_s[kSortBins], tot_s[kSortBins];
+    uint32_t* hist_s = dyn_smem;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t tiles = (k + kSortTile - 1) / kSortTile;
-    const int shift = 8 * pass;
-    grid_dependency_wait();
-    for (uint32_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-        // where each digit's run starts for this tile: all entries of earlier digits, plus
-        // this digit's entries in earlier tiles
-        // (four threads per digit, each over a quarter of the tiles: the chain of dependent loads is what a
-        // pass with many tiles waits for)
-        {
-            const int d = tid & (kSortBins - 1), q = tid / kSortBins;
-            const uint32_t per = (tiles + kParts - 1) / kParts;
-            const uint32_t t_lo = q * per, t_hi = min(tiles, t_lo + per);
-            uint32_t total = 0, bef = 0;
-            for (uint32_t t0 = t_lo; t0 < t_hi; t0 += 8) {
-                uint32_t c[8];
+    const float* __restrict__ losses = p.losses;
+    const int64_t N = p.N;
+    constexpr int64_t kTileElems = int64_t{kThreads} * E;
+    const int64_t tiles_n = (N + kTileElems - 1) / kTileElems;
+    StatusBlock* status = p.ws.status;
+    uint32_t epoch = 0;
+
+    for (int i = tid; i < kSelBins; i += kThreads) hist_s[i] = 0;
+    if (tid < 3) red[tid] = 0;
+    grid_dependency_wait();  // the losses (and the scorer's histogram) are complete from here on
+
+    // the block's first tile stays in registers through all phases of the selection
+    uint32_t key0[E];
+    load_keys<E>(losses, N, static_cast<int64_t>(blockIdx.x) * kTileElems + static_cast<int64_t>(tid) * E, key0);
+    // body(tile, keys) for each of this block's tiles: the first from the registers, any further one reloaded
+    auto for_each_tile = [&](auto&& body) {
+        if (blockIdx.x < tiles_n) body(static_cast<int64_t>(blockIdx.x), key0);
+        for (int64_t tile = static_cast<int64_t>(blockIdx.x) + gridDim.x; tile < tiles_n; tile += gridDim.x) {
+            uint32_t key[E];
+            load_keys<E>(losses, N, tile * kTileElems + static_cast<int64_t>(tid) * E, key);
+            body(tile, key);
+        }
+    };
+
+    // ---- 1. radix select ----
+    uint32_t prefix = 0, want = p.k;
+    if (p.hist0_ready) {
+        uint32_t bin;
+        find_bin(p.ws.hist, kSelBins, want, bin, warp_tot, result);
+        prefix = bin << 21;
+    }
+    for (int pass = p.hist0_ready ? 1 : 0; pass < kSelPasses; ++pass) {
+        const uint32_t mask = prefix_mask(pass);
+        __syncthreads();  // hist_s is zero
+        for_each_tile([&](int64_t, const uint32_t (&key)[E]) {
 #pragma unroll
-                for (int u = 0; u < 8; ++u)  // eight independent loads in flight
-                    c[u] = t0 + u < t_hi ? __ldcg(tile_hist + (t0 + u) * kSortBins + d) : 0u;
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    total += c[u];
-                    bef += t0 + u < tile ? c[u] : 0u;
+            for (int i = 0; i < E; ++i) {
+                const bool in = key[i] != 0u && (key[i] & mask) == prefix;
+                if (pass == 0) {
+                    // every key counts and losses crowd into a few bins: one atomic per distinct digit and warp
+                    const uint32_t d = in ? digit_of(key[i], 0) : 0xFFFFFFFFu;
+                    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, d);
+                    if (in && lane == __ffs(peers) - 1) atomicAdd(&hist_s[d], __popc(peers));
+                } else if (in) {
+                    atomicAdd(&hist_s[digit_of(key[i], pass)], 1u);
                 }
             }
-            part_tot[q][d] = total;
-            part_bef[q][d] = bef;
+        });
+        __syncthreads();
+        uint32_t* gh = p.ws.hist + pass * kSelBins;
+        for (int i = tid; i < kSelBins; i += kThreads) {
+            const uint32_t c = hist_s[i];
+            if (c) atomicAdd(&gh[i], c);
+            hist_s[i] = 0;
         }
+        if (!grid_sync<CLUSTER>(status, epoch)) return;
+        uint32_t bin;
+        find_bin(gh, pass == 2 ? 1024 : kSelBins, want, bin, warp_tot, result);
+        prefix |= pass == 0 ? bin << 21 : pass == 1 ? bin << 10 : bin;
+    }
+    const uint32_t T = prefix, r = want;  // the k-th key, and how many entries equal to it are selected
+
+    // ---- 2. per tile: keys above T, keys equal to T, largest key ----
+    for_each_tile([&](int64_t tile, const uint32_t (&key)[E]) {
+        uint32_t gt = 0, eq = 0, mx = 0;
 #pragma unroll
-        for (int i = 0; i < kWarps * kSortBins / kSortThreads; ++i) (&counters[0][0])[i * kSortThreads + tid] = 0;
-        uint32_t key[kRounds], rank[kRounds];
-        int32_t idx[kRounds];
-        const uint32_t first = tile * kSortTile + warp * (kRounds * 32);
+        for (int i = 0; i < E; ++i) {
+            gt += key[i] > T;
+            eq += key[i] == T;
+            mx = max(mx, key[i]);
+        }
+        uint32_t packed = gt | (eq << 16);  // a tile has at most 16,384 entries
 #pragma unroll
-        for (int rd = 0; rd < kRounds; ++rd) {  // all loads first: they are independent
-            const uint32_t e = first + rd * 32 + lane;
-            key[rd] = e < k ? __ldcg(keys_in + e) : 0u;
-            idx[rd] = e < k ? __ldcg(idx_in + e) : 0;
+        for (int o = 16; o > 0; o >>= 1) {
+            packed += __shfl_xor_sync(0xFFFFFFFFu, packed, o);
+            mx = max(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+        }
+        if (lane == 0) {
+            atomicAdd(&red[0], packed & 0xFFFFu);
+            atomicAdd(&red[1], packed >> 16);
+            atomicMax(&red[2], mx);
         }
         __syncthreads();
-        uint32_t before = 0;
-        if (tid < kSortBins) {
-            uint32_t total = 0;
-#pragma unroll
-            for (int q = 0; q < kParts; ++q) {
-                total += part_tot[q][tid];
-                before += part_bef[q][tid];
-            }
-            tot_s[tid] = total;
+        if (tid == 0) {
+            __stcg(reinterpret_cast<uint4*>(p.ws.tile_counts) + tile, make_uint4(red[0], red[1], red[2], 0u));
+            red[0] = red[1] = red[2] = 0;
         }
         __syncthreads();
-        if (warp == 0) {  // exclusive scan of the 256 digit totals, eight per lane
-            uint32_t v[8], sum = 0;
+    });
+    if (!grid_sync<CLUSTER>(status, epoch)) return;
+
+    // ---- 3. ordered compaction ----
+    // The sort key of a selected entry is u = kmax - key (0 for the largest loss); `passes` 9-bit digits cover its range.
+    uint32_t kmax = 0;
+    for (int64_t t = tid; t < tiles_n; t += kThreads) kmax = max(kmax, __ldcg(p.ws.tile_counts + 4 * t + 2));
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                v[i] = tot_s[lane * 8 + i];
-                sum += v[i];
-            }
-            uint32_t inc = sum;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-                if (lane >= o) inc += n;
-            }
-            uint32_t run = inc - sum;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                tot_s[lane * 8 + i] = run;
-                run += v[i];
-            }
+    for (int o = 16; o > 0; o >>= 1) kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, o));
+    if (lane == 0) atomicMax(&red[2], kmax);
+    __syncthreads();
+    kmax = red[2];
+    __syncthreads();
+    const uint32_t range = kmax - T;
+    const int passes = p.order == LSGD_ORDER_INDEX_ASC ? 0 : (32 - __clz(range) + kSortBits - 1) / kSortBits;
+    const bool direct = passes == 0;  // index order is the final order
+    const int tshift = 10 + (p.sort_rounds == 1 ? 0 : p.sort_rounds == 2 ? 1 : p.sort_rounds == 4 ? 2 : 3);
+    const uint32_t St = p.sort_tiles;
+    for_each_tile([&](int64_t tile, const uint32_t (&key)[E]) {
+        // entries above / equal to the threshold in the tiles before this one
+        if (tid < 2) red[tid] = 0;
+        __syncthreads();
+        uint32_t gt = 0, eq = 0;
+        for (int64_t t = tid; t < tile; t += kThreads) {
+            const uint2 c = __ldcg(reinterpret_cast<const uint2*>(p.ws.tile_counts + 4 * t));
+            gt += c.x;
+            eq += c.y;
         }
 #pragma unroll
-        for (int rd = 0; rd < kRounds; ++rd) {
-            const uint32_t e = first + rd * 32 + lane;
-            const bool live = e < k;
-            const uint32_t dd = 255u - ((key[rd] >> shift) & 0xFFu);
-            const uint32_t peers = match_digit8(dd, live);
-            const int leader = live ? __ffs(peers) - 1 : lane;
-            uint32_t old = 0;
-            if (live && lane == leader) {
-                old = counters[warp][dd];
-                counters[warp][dd] = old + __popc(peers);
-            }
-            old = __shfl_sync(0xFFFFFFFFu, old, leader);
-            rank[rd] = old + __popc(peers & ((1u << lane) - 1u));
-            __syncwarp();
+        for (int o = 16; o > 0; o >>= 1) {
+            gt += __shfl_xor_sync(0xFFFFFFFFu, gt, o);
+            eq += __shfl_xor_sync(0xFFFFFFFFu, eq, o);
+        }
+        if (lane == 0 && (gt | eq)) {
+            atomicAdd(&red[0], gt);
+            atomicAdd(&red[1], eq);
         }
         __syncthreads();
-        if (tid < kSortBins) {
-            base_s[tid] = tot_s[tid] + before;
-            uint32_t run = 0;
+        const uint32_t gt_before = red[0], eq_before = red[1];
+        uint32_t my_gt = 0, my_eq = 0;
 #pragma unroll
-            for (int w = 0; w < kWarps; ++w) {
-                const uint32_t c = counters[w][tid];
-                counters[w][tid] = run;
-                run += c;
-            }
+        for (int i = 0; i < E; ++i) {
+            my_gt += key[i] > T;
+            my_eq += key[i] == T;
         }
-        __syncthreads();
-        if (tile + gridDim.x >= tiles) grid_launch_dependents();  // only this CTA's last scatter is left
+        // one scan for both counts: each is at most 16,384 < 2^16
+        const uint32_t packed = block_exclusive_scan(my_gt | (my_eq << 16), warp_tot);
+        uint32_t gt_run = gt_before + (packed & 0xFFFFu);
+        uint32_t eq_run = eq_before + (packed >> 16);
+        const int64_t base = tile * kTileElems + static_cast<int64_t>(tid) * E;
 #pragma unroll
-        for (int rd = 0; rd < kRounds; ++rd) {
-            const uint32_t e = first + rd * 32 + lane;
-            const bool live = e < k;
-            uint32_t pos = 0;
-            if (live) {
-                const uint32_t dd = 255u - ((key[rd] >> shift) & 0xFFu);
-                pos = base_s[dd] + counters[warp][dd] + rank[rd];
-                idx_out[pos] = idx[rd];
-                if (LAST) {
-                    if (out_vals) out_vals[pos] = losses[idx[rd]];
+        for (int i = 0; i < E; ++i) {
+            const bool above = key[i] > T;
+            const bool tie = key[i] == T;
+            if (above || (tie && eq_run < r)) {
+                const uint32_t pos = gt_run + min(eq_run, r);
+                const int64_t j = base + i;
+                if (direct) {
+                    p.out_idx[pos] = static_cast<int32_t>(j);
+                    if (p.out_vals) p.out_vals[pos] = losses[j];
                 } else {
-                    keys_out[pos] = key[rd];
+                    __stcg(p.ws.idx[0] + pos, static_cast<int32_t>(j));
+                    __stcg(p.ws.keys[0] + pos, key[i]);
+                    atomicAdd(&p.ws.tile_hist[(pos >> tshift) * kSortBins + ((kmax - key[i]) & (kSortBins - 1))], 1u);
                 }
             }
-            if (!LAST) {
-                // count the next digit per destination tile.  High digits are nearly constant over the selection,
-                // so a warp sends one atomic per distinct counter instead of one per entry.
-                const uint32_t nd = 255u - ((key[rd] >> (shift + 8)) & 0xFFu);
-                const uint32_t peers = match_digit8(nd, live);
-                const int leader = live ? __ffs(peers) - 1 : lane;
-                const uint32_t t = pos >> kSortShift;
-                const bool with_leader = t == __shfl_sync(0xFFFFFFFFu, t, leader);  // same destination tile as the leader
-                const uint32_t same = __ballot_sync(0xFFFFFFFFu, live && with_leader);
-                if (live) {
-                    if (lane == leader) atomicAdd(&next_hist[t * kSortBins + nd], static_cast<uint32_t>(__popc(peers & same)));
-                    else if (!with_leader) atomicAdd(&next_hist[t * kSortBins + nd], 1u);
-                }
-            }
+            gt_run += above;
+            eq_run += tie;
         }
         __syncthreads();
+    });
+    if (direct) return;
+    if (!grid_sync<CLUSTER>(status, epoch)) return;
+
+    // ---- 4. stable LSD sort of the k pairs on u = kmax - key, ascending, 9 bits per pass ----
+    uint32_t(*counters)[kCounterPitch] = reinterpret_cast<uint32_t(*)[kCounterPitch]>(dyn_smem);
+    const int R = p.sort_rounds;
+    const uint32_t k = p.k;
+    for (int pass = 0; pass < passes; ++pass) {
+        const bool last = pass == passes - 1;
+        const int shift = kSortBits * pass;
+        const uint32_t* keys_in = p.ws.keys[pass & 1];
+        const int32_t* idx_in = p.ws.idx[pass & 1];
+        uint32_t* keys_out = p.ws.keys[(pass + 1) & 1];
+        int32_t* idx_out = last ? p.out_idx : p.ws.idx[(pass + 1) & 1];
+        const uint32_t* cnt = p.ws.tile_hist + static_cast<size_t>(pass) * p.ws.pass_stride;
+        uint32_t* cnt_next = p.ws.tile_hist + static_cast<size_t>(pass + 1) * p.ws.pass_stride;
+        for (uint32_t tile = blockIdx.x; tile < St; tile += gridDim.x) {
+            // where each digit's run starts for this tile: all entries of smaller digits, plus this digit's
+            // entries in earlier tiles (two threads per digit, each over half of the tiles)
+            {
+                const int d = tid & (kSortBins - 1), q = tid / kSortBins;
+                const uint32_t per = (St + 1) / 2;
+                const uint32_t t_lo = q * per, t_hi = min(St, t_lo + per);
+                uint32_t total = 0, bef = 0;
+                for (uint32_t t0 = t_lo; t0 < t_hi; t0 += 16) {
+                    uint32_t c[16];
+#pragma unroll
+                    for (int u = 0; u < 16; ++u)  // sixteen independent loads in flight
+                        c[u] = t0 + u < t_hi ? __ldcg(cnt + static_cast<size_t>(t0 + u) * kSortBins + d) : 0u;
+#pragma unroll
+                    for (int u = 0; u < 16; ++u) {
+                        total += c[u];
+                        bef += t0 + u < tile ? c[u] : 0u;
+                    }
+                }
+                part_tot[q][d] = total;
+                part_bef[q][d] = bef;
+            }
+            for (int i = tid; i < kWarps * kCounterPitch; i += kThreads) dyn_smem[i] = 0;
+            uint32_t key[kSortMaxRounds], rank[kSortMaxRounds];
+            int32_t idx[kSortMaxRounds];
+            const uint32_t first = (tile << tshift) + warp * (R * 32);
+#pragma unroll
+            for (int rd = 0; rd < kSortMaxRounds; ++rd) {  // all loads first: they are independent
+                const uint32_t e = first + rd * 32 + lane;
+                const bool live = rd < R && e < k;
+                key[rd] = live ? __ldcg(keys_in + e) : 0u;
+                idx[rd] = live ? __ldcg(idx_in + e) : 0;
+            }
+            __syncthreads();
+            uint32_t before = 0;
+            if (tid < kSortBins) {
+                before = part_bef[0][tid] + part_bef[1][tid];
+                tot_s[tid] = part_tot[0][tid] + part_tot[1][tid];
+            }
+            __syncthreads();
+            if (warp == 0) {  // exclusive scan of the 512 digit totals, sixteen per lane
+                constexpr int kPer = kSortBins / 32;
+                uint32_t v[kPer], sum = 0;
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) {
+                    v[i] = tot_s[lane * kPer + i];
+                    sum += v[i];
+                }
+                uint32_t inc = sum;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                    if (lane >= o) inc += n;
+                }
+                uint32_t run = inc - sum;
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) {
+                    tot_s[lane * kPer + i] = run;
+                    run += v[i];
+                }
+            }
+            // stable rank inside the warp's run of entries (rounds in order, lanes in order)
+#pragma unroll
+            for (int rd = 0; rd < kSortMaxRounds; ++rd) {
+                if (rd < R) {
+                    const uint32_t e = first + rd * 32 + lane;
+                    const bool live = e < k;
+                    const uint32_t dd = ((kmax - key[rd]) >> shift) & (kSortBins - 1);
+                    const uint32_t peers = match_digit(dd, live);
+                    const int leader = live ? __ffs(peers) - 1 : lane;
+                    uint32_t old = 0;
+                    if (live && lane == leader) {
+                        old = counters[warp][dd];
+                        counters[warp][dd] = old + __popc(peers);
+                    }
+                    old = __shfl_sync(0xFFFFFFFFu, old, leader);
+                    rank[rd] = old + __popc(peers & ((1u << lane) - 1u));
+                    __syncwarp();
+                }
+            }
+            __syncthreads();
+            if (tid < kSortBins) base_s[tid] = tot_s[tid] + before;
+            // per digit, exclusive prefix of the warps' counts: one warp per 16 digits, lane = source warp
+#pragma unroll 4
+            for (int i = 0; i < kSortBins / kWarps; ++i) {
+                const int d = warp * (kSortBins / kWarps) + i;
+                const uint32_t c = counters[lane][d];
+                uint32_t inc = c;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                    if (lane >= o) inc += n;
+                }
+                counters[lane][d] = inc - c;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int rd = 0; rd < kSortMaxRounds; ++rd) {
+                if (rd < R) {
+                    const uint32_t e = first + rd * 32 + lane;
+                    const bool live = e < k;
+                    uint32_t pos = 0;
+                    if (live) {
+                        const uint32_t dd = ((kmax - key[rd]) >> shift) & (kSortBins - 1);
+                        pos = base_s[dd] + counters[warp][dd] + rank[rd];
+                        if (last) {
+                            idx_out[pos] = idx[rd];
+                            if (p.out_vals) p.out_vals[pos] = losses[idx[rd]];
+                        } else {
+                            __stcg(idx_out + pos, idx[rd]);
+                            __stcg(keys_out + pos, key[rd]);
+                        }
+                    }
+                    if (!last) {
+                        // count the next digit per destination tile.  High digits are nearly constant over the
+                        // selection, so a warp sends one atomic per distinct counter instead of one per entry.
+                        const uint32_t nd = ((kmax - key[rd]) >> (shift + kSortBits)) & (kSortBins - 1);
+                        const uint32_t peers = match_digit(nd, live);
+                        const int leader = live ? __ffs(peers) - 1 : lane;
+                        const uint32_t t = pos >> tshift;
+                        const bool with_leader = t == __shfl_sync(0xFFFFFFFFu, t, leader);  // same destination tile as the leader
+                        const uint32_t same = __ballot_sync(0xFFFFFFFFu, live && with_leader);
+                        if (live) {
+                            if (lane == leader) atomicAdd(&cnt_next[static_cast<size_t>(t) * kSortBins + nd], static_cast<uint32_t>(__popc(peers & same)));
+                            else if (!with_leader) atomicAdd(&cnt_next[static_cast<size_t>(t) * kSortBins + nd], 1u);
+                        }
+                    }
+                }
+            }
+            __syncthreads();
+        }
+        if (!last && !grid_sync<CLUSTER>(status, epoch)) return;
     }
 }
 
@@ -595,18 +620,10 @@ small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int
     }
     // index-ascending: an entry is selected iff its composite key is >= the k-th largest
     const unsigned long long cut = ck[k - 1];
-    constexpr int kPer = 1;  // one index per thread
-    const int base = threadIdx.x * kPer;
-    bool sel[kPer];
-    uint32_t mine = 0;
-#pragma unroll
-    for (int i = 0; i < kPer; ++i) {
-        const int j = base + i;
-        sel[i] = j < n && ((static_cast<unsigned long long>(loss_key(losses[j])) << 32) | (0xFFFFFFFFu - static_cast<uint32_t>(j))) >= cut;
-        mine += sel[i];
-    }
+    const int j = threadIdx.x;  // one index per thread
+    const bool sel = j < n && ((static_cast<unsigned long long>(loss_key(losses[j])) << 32) | (0xFFFFFFFFu - static_cast<uint32_t>(j))) >= cut;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t inc = mine;
+    uint32_t inc = sel;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, inc, o);
@@ -614,15 +631,59 @@ small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int
     }
     if (lane == 31) warp_tot[warp] = inc;
     __syncthreads();
-    uint32_t pos = inc - mine;
+    uint32_t pos = inc - sel;
     for (int w = 0; w < warp; ++w) pos += warp_tot[w];
-#pragma unroll
-    for (int i = 0; i < kPer; ++i)
-        if (sel[i]) {
-            out_idx[pos] = base + i;
-            if (out_vals) out_vals[pos] = losses[base + i];
-            ++pos;
-        }
+    if (sel) {
+        out_idx[pos] = j;
+        if (out_vals) out_vals[pos] = losses[j];
+    }
+}
+
+template <int E, bool CLUSTER>
+cudaError_t launch_select(const SelectParams& p, int grid, cudaStream_t s) {
+    auto kernel = topk_select_kernel<E, CLUSTER>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kDynSmemBytes));
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kDynSmemBytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    if (CLUSTER) {
+        // one cluster; it may be scheduled while the previous kernel of the stream drains (it waits for that
+        // kernel's completion before its first global access)
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = static_cast<unsigned>(grid);
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.numAttrs = 2;
+    } else {
+        attr[0].id = cudaLaunchAttributeCooperative;  // all blocks resident at once, or the launch is refused
+        attr[0].val.cooperative = 1;
+        cfg.numAttrs = 1;
+    }
+    cfg.attrs = attr;
+    return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
+// Blocks of topk_select_kernel that can be resident at once on the current device (cached per device).
+int resident_blocks() {
+    static int cache[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 1;
+    int& c = cache[dev & 63];
+    if (c == 0) {
+        auto kernel = topk_select_kernel<16, false>;
+        int per_sm = 0;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kDynSmemBytes)) != cudaSuccess ||
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, kDynSmemBytes) != cudaSuccess || per_sm < 1)
+            per_sm = 1;
+        c = sm_count() * per_sm;
+    }
+    return c;
 }
 
 }  // namespace
@@ -632,37 +693,34 @@ cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order or
     if (N <= kSmallN)
         return launch_dependent(small_topk_kernel, 1, kSmallThreads, s, losses, static_cast<int>(N), static_cast<int>(k),
                                 static_cast<int>(order), out_idx, out_vals);
-    const int64_t tiles_n = (N + kTile - 1) / kTile;
-    const int grid_n = static_cast<int>(std::min<int64_t>(tiles_n, static_cast<int64_t>(sm_count()) * 8));
-    const uint32_t kk = static_cast<uint32_t>(k);
-    cudaError_t e = cudaSuccess;
-    for (int pass = hist0_ready ? 1 : 0; pass < kSelPasses && e == cudaSuccess; ++pass)
-        e = launch_dependent(select_hist_kernel, grid_n, kThreads, s, losses, N, kk, pass,
-                             pass > (hist0_ready ? 1 : 0), ws.hist, ws.status);
-    if (e != cudaSuccess) return e;
-    e = launch_dependent(select_count_kernel, grid_n, kThreads, s, losses, N, ws.status, ws.tile_counts);
-    if (e != cudaSuccess) return e;
-    if (order == LSGD_ORDER_INDEX_ASC)
-        return launch_dependent(select_emit_kernel<true>, grid_n, kThreads, s, losses, N, ws.status, ws.tile_counts,
-                                out_idx, out_vals, nullptr, nullptr, 12);
-    const int sort_shift = sort_tile_shift(k);
-    const int64_t tiles_k = static_cast<int64_t>(sort_tiles(k));
-    const size_t th = sort_tiles_bound(k) * kSortBins;  // digit counts of one pass
-    e = launch_dependent(select_emit_kernel<false>, grid_n, kThreads, s, losses, N, ws.status, ws.tile_counts, ws.idx[0],
-                         nullptr, ws.keys[0], ws.tile_hist, sort_shift);
-    const int grid_k = static_cast<int>(std::min<int64_t>(tiles_k, static_cast<int64_t>(sm_count()) * 2));
-    auto pass_kernel = [&](auto mid, auto last) {
-        for (int pass = 0; pass < 3 && e == cudaSuccess; ++pass)
-            e = launch_dependent(mid, grid_k, kSortThreads, s, ws.keys[pass & 1], ws.idx[pass & 1], kk, pass,
-                                 ws.tile_hist + pass * th, ws.keys[(pass + 1) & 1], ws.idx[(pass + 1) & 1],
-                                 ws.tile_hist + (pass + 1) * th, nullptr, nullptr);
-        if (e != cudaSuccess) return;
-        e = launch_dependent(last, grid_k, kSortThreads, s, ws.keys[1], ws.idx[1], kk, 3, ws.tile_hist + 3 * th, nullptr,
-                             out_idx, nullptr, losses, out_vals);
-    };
-    if (sort_shift == 10) pass_kernel(sort_scatter_kernel<false, 1>, sort_scatter_kernel<true, 1>);
-    else pass_kernel(sort_scatter_kernel<false, 4>, sort_scatter_kernel<true, 4>);
-    return e;
+    SelectParams p;
+    p.losses = losses;
+    p.N = N;
+    p.k = static_cast<uint32_t>(k);
+    p.order = static_cast<int>(order);
+    p.out_idx = out_idx;
+    p.out_vals = out_vals;
+    p.ws = ws;
+    p.hist0_ready = hist0_ready ? 1 : 0;
+    const TestGeometry tg = test_geometry();
+    // One cluster of up to 8 blocks, 8,192 entries each, when the pool fits.
+    constexpr int64_t kClusterTile = int64_t{kThreads} * 8;
+    const int max_cluster = std::max(1, std::min(kMaxClusterBlocks, tg.max_ctas));
+    if (!tg.no_cluster && N <= kClusterTile * kMaxClusterBlocks) {
+        const int grid = static_cast<int>(std::min<int64_t>((N + kClusterTile - 1) / kClusterTile, max_cluster));
+        p.sort_rounds = sort_rounds_for(k, grid);
+        p.sort_tiles = static_cast<uint32_t>((k + 1024 * p.sort_rounds - 1) / (1024 * p.sort_rounds));
+        return launch_select<8, true>(p, grid, s);
+    }
+    const int resident = std::max(1, std::min(resident_blocks(), tg.max_ctas));
+    p.sort_rounds = sort_rounds_for(k, std::min(resident, kSortDirectTiles));
+    p.sort_tiles = static_cast<uint32_t>((k + 1024 * p.sort_rounds - 1) / (1024 * p.sort_rounds));
+    auto tiles = [&](int e) { return (N + int64_t{kThreads} * e - 1) / (int64_t{kThreads} * e); };
+    const int e = tiles(4) <= resident ? 4 : tiles(8) <= resident ? 8 : 16;
+    const int grid = static_cast<int>(std::min<int64_t>(resident, std::max<int64_t>(tiles(e), p.sort_tiles)));
+    if (e == 4) return launch_select<4, false>(p, grid, s);
+    if (e == 8) return launch_select<8, false>(p, grid, s);
+    return launch_select<16, false>(p, grid, s);
 }
 
 }  // namespace lsgd

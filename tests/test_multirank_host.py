@@ -51,4 +51,5 @@ def test_bench_accounting_helpers():
     assert b == (cfg.N - 100) * (cfg.C * 4 + 4) + cfg.N * 8 + 8 * cfg.N + 8 * cfg.k
     assert bench.aggregate_bytes(cfg) == 4 * cfg.D * (cfg.P + 1)
     assert bench.launches_per_step(wl.CONFIGS[4]) == 1 + 1 + 1 + 1
-    assert bench.launches_per_step(wl.CONFIGS[5]) == 1 + 2 + 1 + 1 + 4 + 1
+    assert bench.launches_per_step(wl.CONFIGS[5]) == 1 + 1 + 1
+    assert bench.launches_per_step(wl.CONFIGS[1]) == 1 + 1 + 1 + 1  # D = 272,474 leaves a ragged tail
