@@ -3,9 +3,14 @@
 // One pass over P + 1 streams: every thread owns one 16-byte column slice at a
 // time, issues the P replica loads back to back (P independent 128-bit loads in
 // flight per thread), folds them in ascending i with one multiply and P - 1 fused
-// multiply-adds, and stores once.  All traffic is marked streaming: nothing is
-// read twice, so nothing should stay in L1 or linger in L2.  The kernel is bound
-// by HBM bandwidth: 4 (P + 1) bytes per parameter.
+// multiply-adds, and stores once.  Loads go past L1 (ld.global.cg) with the
+// normal L2 policy, stores are marked evict-first.  Evict-first LOADS
+// (ld.global.cs) were 11 % slower whenever the L2 still held lines of some other
+// buffer written earlier with the normal policy (any real program): such lines
+// are never displaced by evict-first traffic, which then has to make do with
+// what is left of the L2 (measured: 760 us instead of 687 us for 10 x 109 M
+// parameters, in every state but a freshly started process).  The kernel is
+// bound by HBM bandwidth: 4 (P + 1) bytes per parameter.
 #include "lsgd_internal.cuh"
 
 namespace lsgd {
@@ -41,7 +46,7 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_vec4_kernel(const __gri
         if constexpr (PCT > 0) {
             float4 v[PCT];
 #pragma unroll
-            for (int r = 0; r < PCT; ++r) v[r] = __ldcs(reinterpret_cast<const float4*>(a.x[r]) + i);
+            for (int r = 0; r < PCT; ++r) v[r] = __ldcg(reinterpret_cast<const float4*>(a.x[r]) + i);
             acc = mul4(a.w[0], v[0]);
 #pragma unroll
             for (int r = 1; r < PCT; ++r) acc = fma4(a.w[r], v[r], acc);
@@ -51,7 +56,7 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_vec4_kernel(const __gri
                 float4 v[kAggBatch];
 #pragma unroll
                 for (int u = 0; u < kAggBatch; ++u)
-                    if (b + u < P) v[u] = __ldcs(reinterpret_cast<const float4*>(a.x[b + u]) + i);
+                    if (b + u < P) v[u] = __ldcg(reinterpret_cast<const float4*>(a.x[b + u]) + i);
 #pragma unroll
                 for (int u = 0; u < kAggBatch; ++u)
                     if (b + u < P) acc = (b + u == 0) ? mul4(a.w[0], v[u]) : fma4(a.w[b + u], v[u], acc);
@@ -68,8 +73,8 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_scalar_kernel(const __g
                                                                         float* out) {
     const int64_t stride = static_cast<int64_t>(gridDim.x) * kAggThreads;
     for (int64_t j = begin + static_cast<int64_t>(blockIdx.x) * kAggThreads + threadIdx.x; j < D; j += stride) {
-        float acc = a.w[0] * __ldcs(a.x[0] + j);
-        for (int r = 1; r < P; ++r) acc = fmaf(a.w[r], __ldcs(a.x[r] + j), acc);
+        float acc = a.w[0] * __ldcg(a.x[0] + j);
+        for (int r = 1; r < P; ++r) acc = fmaf(a.w[r], __ldcg(a.x[r] + j), acc);
         out[j] = acc;
     }
 }

@@ -39,7 +39,7 @@ struct Slice<float> {
     __device__ __forceinline__ static void store(void* p, int64_t i, const float (&r)[4]) {
         __stcs(reinterpret_cast<float4*>(p) + i, make_float4(r[0], r[1], r[2], r[3]));
     }
-    __device__ __forceinline__ static float load_one(const void* p, int64_t j) { return __ldcs(static_cast<const float*>(p) + j); }
+    __device__ __forceinline__ static float load_one(const void* p, int64_t j) { return __ldcg(static_cast<const float*>(p) + j); }
     __device__ __forceinline__ static void store_one(void* p, int64_t j, float r) { static_cast<float*>(p)[j] = r; }
 };
 
@@ -81,7 +81,7 @@ aggregate_round_kernel(const __grid_constant__ RoundArgs a, int P, int64_t n_sli
         if (BASE) {
 #pragma unroll
             for (int q = 0; q < E / 4; ++q) {
-                const float4 t = __ldcs(reinterpret_cast<const float4*>(base) + i * (E / 4) + q);
+                const float4 t = __ldcg(reinterpret_cast<const float4*>(base) + i * (E / 4) + q);
                 b[4 * q] = t.x; b[4 * q + 1] = t.y; b[4 * q + 2] = t.z; b[4 * q + 3] = t.w;
             }
         }
@@ -89,7 +89,7 @@ aggregate_round_kernel(const __grid_constant__ RoundArgs a, int P, int64_t n_sli
             uint4 raw[kBatch];
 #pragma unroll
             for (int u = 0; u < kBatch; ++u)
-                if (r0 + u < P) raw[u] = __ldcs(reinterpret_cast<const uint4*>(a.x[r0 + u]) + i);
+                if (r0 + u < P) raw[u] = __ldcg(reinterpret_cast<const uint4*>(a.x[r0 + u]) + i);
 #pragma unroll
             for (int u = 0; u < kBatch; ++u)
                 if (r0 + u < P) {

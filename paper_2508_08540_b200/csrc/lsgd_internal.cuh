@@ -38,17 +38,15 @@ constexpr int kSortBits = 9;              // digits of the stable LSD sort of th
 constexpr int kSortBins = 1 << kSortBits;
 constexpr int kSortPasses = 4;            // at most: 4 x 9 bits cover a 32-bit key range
 constexpr int kSortMaxRounds = 8;         // a sort tile holds 1024 R entries, R in {1, 2, 4, 8}
-constexpr int kSortDirectTiles = 64;      // the launcher grows R before it uses more sort tiles than this
+constexpr int kSortDirectTiles = 256;     // the launcher grows R before it uses more sort tiles than this
 constexpr int kMaxClusterBlocks = 8;      // portable cluster size: pools of up to 8 x 8,192 entries run as one cluster
 
 struct TopkWorkspace {       // device pointers carved out of the caller's workspace
     StatusBlock* status;
     uint32_t* hist;          // [kSelPasses][kSelBins]
     uint32_t* tile_counts;   // [tiles(N)][4]  (#keys above the threshold, #keys equal to it, largest key, unused)
-    uint32_t* keys[2];       // [k] ping-pong: keys of the selected entries
-    int32_t* idx[2];         // [k] ping-pong: their indices
-    uint32_t* tile_hist;     // [kSortPasses][sort tiles][kSortBins] digit counts per sort tile and pass
-    uint32_t pass_stride;    // words between the digit counts of consecutive passes
+    uint2* pairs[2];         // [k] ping-pong: (key, index) of the selected entries
+    uint32_t* tile_hist;     // [sort tiles][kSortBins] digit counts per sort tile of the current pass
 };
 
 // Test hooks (environment, read at every launch): they change launch geometry only, never results.

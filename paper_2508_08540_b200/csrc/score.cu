@@ -608,13 +608,13 @@ score_stream_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int v = v_begin + u * 32 + lane;
-                raw[u] = v < v_end ? __ldcs(vbase + v) : none;
+                raw[u] = v < v_end ? __ldcg(vbase + v) : none;
             }
             for (int v0 = v_begin; v0 < v_end; v0 += 32 * U) {
 #pragma unroll
                 for (int u = 0; u < U; ++u) {  // the next step's vectors
                     const int v = v0 + 32 * U + u * 32 + lane;
-                    nxt[u] = v < v_end ? __ldcs(vbase + v) : none;
+                    nxt[u] = v < v_end ? __ldcg(vbase + v) : none;
                 }
 #pragma unroll
                 for (int u = 0; u < U; ++u)

@@ -24,7 +24,7 @@ constexpr size_t kMaxSortTiles = kSortDirectTiles;  // pools of this size never 
 static_assert(kMaxN <= size_t{kSortDirectTiles} * 1024 * kSortMaxRounds, "the sort's tile bound covers the largest pool");
 constexpr size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 constexpr size_t kScratchBytes = sizeof(StatusBlock) + up256(sizeof(uint32_t) * kSelPasses * kSelBins) +
-                                 up256(sizeof(uint32_t) * kSortPasses * kMaxSortTiles * kSortBins) +
+                                 up256(sizeof(uint32_t) * kMaxSortTiles * kSortBins) +
                                  up256(sizeof(uint32_t) * 4 * kMaxTiles) + 4 * up256(sizeof(uint32_t) * kMaxN);
 
 // The scratch itself.  In host code this name is only a handle for the runtime's

@@ -19,8 +19,8 @@
 //      pairs on u = (largest key - key) in 9-bit digits: only as many passes as
 //      u's range needs (three for losses that span up to 16 binades above T, none
 //      if all selected keys are equal); stability turns the index-ascending input
-//      order into the required tie-break.  Each scatter counts the next digit per
-//      destination tile, so a pass is one phase.
+//      order into the required tie-break.  A pass is two phases: rank every tile
+//      by the digit (which gives the tile's digit counts), then scatter.
 // The kernel runs either as ONE thread-block cluster (pools of up to 65,536
 // entries: the barrier is the cluster's hardware barrier) or as a cooperative
 // launch with one block per multiprocessor (all blocks resident by construction;
@@ -49,7 +49,7 @@ static size_t sort_tiles_bound(int64_t k) {
     if (k <= int64_t{kSortDirectTiles} * 1024 * kSortMaxRounds) return static_cast<size_t>(std::min<int64_t>(kSortDirectTiles, (k + 1023) / 1024));
     return static_cast<size_t>((k + 1024 * kSortMaxRounds - 1) / (1024 * kSortMaxRounds));
 }
-static size_t sort_count_words(int64_t k) { return static_cast<size_t>(kSortPasses) * sort_tiles_bound(k) * kSortBins; }
+static size_t sort_count_words(int64_t k) { return sort_tiles_bound(k) * kSortBins; }
 
 size_t topk_workspace_bytes(int64_t N, int64_t k) {
     if (N < 0 || k < 0 || k > N) return 0;
@@ -62,11 +62,9 @@ size_t topk_workspace_bytes(int64_t N, int64_t k) {
     return b;
 }
 
-// Bytes at the start of the workspace that one memset must clear before a call.
-static size_t topk_zero_bytes(int64_t k) {
-    return sizeof(StatusBlock) + align_up(sizeof(uint32_t) * kSelPasses * kSelBins) +
-           align_up(sizeof(uint32_t) * sort_count_words(k));
-}
+// Bytes at the start of the workspace that one memset must clear before a call: the status block and the
+// selection's digit histograms.
+static size_t topk_zero_bytes(int64_t) { return sizeof(StatusBlock) + align_up(sizeof(uint32_t) * kSelPasses * kSelBins); }
 
 TopkWorkspace carve_topk(void* ws, int64_t N, int64_t k) {
     const size_t tiles_n = static_cast<size_t>((N + kTile - 1) / kTile);
@@ -77,15 +75,12 @@ TopkWorkspace carve_topk(void* ws, int64_t N, int64_t k) {
     w.hist = reinterpret_cast<uint32_t*>(p);
     p += align_up(sizeof(uint32_t) * kSelPasses * kSelBins);
     w.tile_hist = reinterpret_cast<uint32_t*>(p);
-    w.pass_stride = static_cast<uint32_t>(sort_tiles_bound(k) * kSortBins);
     p += align_up(sizeof(uint32_t) * sort_count_words(k));
     w.tile_counts = reinterpret_cast<uint32_t*>(p);
     p += align_up(sizeof(uint32_t) * 4 * tiles_n);
     const size_t kb = align_up(sizeof(uint32_t) * static_cast<size_t>(k));
-    w.keys[0] = reinterpret_cast<uint32_t*>(p);
-    w.keys[1] = reinterpret_cast<uint32_t*>(p + kb);
-    w.idx[0] = reinterpret_cast<int32_t*>(p + 2 * kb);
-    w.idx[1] = reinterpret_cast<int32_t*>(p + 3 * kb);
+    w.pairs[0] = reinterpret_cast<uint2*>(p);
+    w.pairs[1] = reinterpret_cast<uint2*>(p + 2 * kb);
     return w;
 }
 
@@ -253,7 +248,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
     __shared__ uint32_t result[2];
     __shared__ uint32_t red[3];
     __shared__ uint32_t part_tot[2][kSortBins], part_bef[2][kSortBins];
-    __shared__ uint32_t base_s[kSortBins], tot_s[kSortBins];
+    __shared__ uint32_t base_s[kSortBins], tot_s[kSortBins], half_cnt[2][kSortBins];
     uint32_t* hist_s = dyn_smem;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float* __restrict__ losses = p.losses;
@@ -405,9 +400,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
                     p.out_idx[pos] = static_cast<int32_t>(j);
                     if (p.out_vals) p.out_vals[pos] = losses[j];
                 } else {
-                    __stcg(p.ws.idx[0] + pos, static_cast<int32_t>(j));
-                    __stcg(p.ws.keys[0] + pos, key[i]);
-                    atomicAdd(&p.ws.tile_hist[(pos >> tshift) * kSortBins + ((kmax - key[i]) & (kSortBins - 1))], 1u);
+                    __stcg(p.ws.pairs[0] + pos, make_uint2(key[i], static_cast<uint32_t>(j)));
                 }
             }
             gt_run += above;
@@ -419,19 +412,87 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
     if (!grid_sync<CLUSTER>(status, epoch)) return;
 
     // ---- 4. stable LSD sort of the k pairs on u = kmax - key, ascending, 9 bits per pass ----
+    // A pass has two halves with a barrier between them: every tile ranks its entries by the pass's digit
+    // (which also yields the tile's digit counts, written to tile_hist); then every tile reads all tiles' counts,
+    // derives where its runs start, and scatters.  A block with a single tile keeps its ranks in registers and
+    // shared memory across the barrier; a block with several tiles ranks each of them a second time.
     uint32_t(*counters)[kCounterPitch] = reinterpret_cast<uint32_t(*)[kCounterPitch]>(dyn_smem);
     const int R = p.sort_rounds;
     const uint32_t k = p.k;
+    const bool one_tile = St <= gridDim.x;
+    uint32_t key[kSortMaxRounds], rank[kSortMaxRounds];
+    int32_t idx[kSortMaxRounds];
     for (int pass = 0; pass < passes; ++pass) {
         const bool last = pass == passes - 1;
         const int shift = kSortBits * pass;
-        const uint32_t* keys_in = p.ws.keys[pass & 1];
-        const int32_t* idx_in = p.ws.idx[pass & 1];
-        uint32_t* keys_out = p.ws.keys[(pass + 1) & 1];
-        int32_t* idx_out = last ? p.out_idx : p.ws.idx[(pass + 1) & 1];
-        const uint32_t* cnt = p.ws.tile_hist + static_cast<size_t>(pass) * p.ws.pass_stride;
-        uint32_t* cnt_next = p.ws.tile_hist + static_cast<size_t>(pass + 1) * p.ws.pass_stride;
+        const uint2* pairs_in = p.ws.pairs[pass & 1];
+        uint2* pairs_out = p.ws.pairs[(pass + 1) & 1];
+        uint32_t* cnt = p.ws.tile_hist;  // [St][kSortBins], rewritten by every pass
+
+        // Loads a tile, ranks its entries stably by this pass's digit: afterwards rank[rd] is the entry's rank
+        // among the entries of its warp with the same digit, counters[w][d] the number of such entries in the
+        // warps before w of the same half of the block, half_cnt[h][d] the count of half h.
+        auto rank_tile = [&](uint32_t tile, bool publish) {
+            for (int i = tid; i < kWarps * kCounterPitch; i += kThreads) dyn_smem[i] = 0;
+            const uint32_t first = (tile << tshift) + warp * (R * 32);
+#pragma unroll
+            for (int rd = 0; rd < kSortMaxRounds; ++rd) {  // all loads first: they are independent
+                const uint32_t e = first + rd * 32 + lane;
+                const bool live = rd < R && e < k;
+                const uint2 pr = live ? __ldcg(pairs_in + e) : make_uint2(0u, 0u);
+                key[rd] = pr.x;
+                idx[rd] = static_cast<int32_t>(pr.y);
+            }
+            __syncthreads();
+#pragma unroll
+            for (int rd = 0; rd < kSortMaxRounds; ++rd) {
+                if (rd < R) {
+                    const uint32_t e = first + rd * 32 + lane;
+                    const bool live = e < k;
+                    const uint32_t dd = ((kmax - key[rd]) >> shift) & (kSortBins - 1);
+                    const uint32_t peers = match_digit(dd, live);
+                    const int leader = live ? __ffs(peers) - 1 : lane;
+                    uint32_t old = 0;
+                    if (live && lane == leader) {
+                        old = counters[warp][dd];
+                        counters[warp][dd] = old + __popc(peers);
+                    }
+                    old = __shfl_sync(0xFFFFFFFFu, old, leader);
+                    rank[rd] = old + __popc(peers & ((1u << lane) - 1u));
+                    __syncwarp();
+                }
+            }
+            __syncthreads();
+            {   // per digit, exclusive prefix of the warps' counts within each half of the block: thread (digit, half)
+                const int d = tid & (kSortBins - 1), h = tid / kSortBins;
+                constexpr int kHalf = kWarps / 2;
+                uint32_t c[kHalf];
+#pragma unroll
+                for (int u = 0; u < kHalf; ++u) c[u] = counters[kHalf * h + u][d];
+                uint32_t run = 0;
+#pragma unroll
+                for (int u = 0; u < kHalf; ++u) {
+                    counters[kHalf * h + u][d] = run;
+                    run += c[u];
+                }
+                half_cnt[h][d] = run;
+            }
+            __syncthreads();
+            if (publish && tid < kSortBins) __stcg(cnt + static_cast<size_t>(tile) * kSortBins + tid, half_cnt[0][tid] + half_cnt[1][tid]);
+        };
+
+        if (one_tile) {
+            if (blockIdx.x < St) rank_tile(blockIdx.x, true);
+        } else {
+            for (uint32_t tile = blockIdx.x; tile < St; tile += gridDim.x) rank_tile(tile, true);
+        }
+        if (!grid_sync<CLUSTER>(status, epoch)) return;
+
         for (uint32_t tile = blockIdx.x; tile < St; tile += gridDim.x) {
+            if (!one_tile) {
+                __syncthreads();
+                rank_tile(tile, false);
+            }
             // where each digit's run starts for this tile: all entries of smaller digits, plus this digit's
             // entries in earlier tiles (two threads per digit, each over half of the tiles)
             {
@@ -452,17 +513,6 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
                 }
                 part_tot[q][d] = total;
                 part_bef[q][d] = bef;
-            }
-            for (int i = tid; i < kWarps * kCounterPitch; i += kThreads) dyn_smem[i] = 0;
-            uint32_t key[kSortMaxRounds], rank[kSortMaxRounds];
-            int32_t idx[kSortMaxRounds];
-            const uint32_t first = (tile << tshift) + warp * (R * 32);
-#pragma unroll
-            for (int rd = 0; rd < kSortMaxRounds; ++rd) {  // all loads first: they are independent
-                const uint32_t e = first + rd * 32 + lane;
-                const bool live = rd < R && e < k;
-                key[rd] = live ? __ldcg(keys_in + e) : 0u;
-                idx[rd] = live ? __ldcg(idx_in + e) : 0;
             }
             __syncthreads();
             uint32_t before = 0;
@@ -492,75 +542,26 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
                     run += v[i];
                 }
             }
-            // stable rank inside the warp's run of entries (rounds in order, lanes in order)
-#pragma unroll
-            for (int rd = 0; rd < kSortMaxRounds; ++rd) {
-                if (rd < R) {
-                    const uint32_t e = first + rd * 32 + lane;
-                    const bool live = e < k;
-                    const uint32_t dd = ((kmax - key[rd]) >> shift) & (kSortBins - 1);
-                    const uint32_t peers = match_digit(dd, live);
-                    const int leader = live ? __ffs(peers) - 1 : lane;
-                    uint32_t old = 0;
-                    if (live && lane == leader) {
-                        old = counters[warp][dd];
-                        counters[warp][dd] = old + __popc(peers);
-                    }
-                    old = __shfl_sync(0xFFFFFFFFu, old, leader);
-                    rank[rd] = old + __popc(peers & ((1u << lane) - 1u));
-                    __syncwarp();
-                }
-            }
             __syncthreads();
             if (tid < kSortBins) base_s[tid] = tot_s[tid] + before;
-            // per digit, exclusive prefix of the warps' counts: one warp per 16 digits, lane = source warp
-#pragma unroll 4
-            for (int i = 0; i < kSortBins / kWarps; ++i) {
-                const int d = warp * (kSortBins / kWarps) + i;
-                const uint32_t c = counters[lane][d];
-                uint32_t inc = c;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-                    if (lane >= o) inc += n;
-                }
-                counters[lane][d] = inc - c;
-            }
             __syncthreads();
+            const uint32_t first = (tile << tshift) + warp * (R * 32);
 #pragma unroll
             for (int rd = 0; rd < kSortMaxRounds; ++rd) {
                 if (rd < R) {
                     const uint32_t e = first + rd * 32 + lane;
-                    const bool live = e < k;
-                    uint32_t pos = 0;
-                    if (live) {
+                    if (e < k) {
                         const uint32_t dd = ((kmax - key[rd]) >> shift) & (kSortBins - 1);
-                        pos = base_s[dd] + counters[warp][dd] + rank[rd];
+                        const uint32_t pos = base_s[dd] + counters[warp][dd] + (warp >= kWarps / 2 ? half_cnt[0][dd] : 0u) + rank[rd];
                         if (last) {
-                            idx_out[pos] = idx[rd];
+                            p.out_idx[pos] = idx[rd];
                             if (p.out_vals) p.out_vals[pos] = losses[idx[rd]];
                         } else {
-                            __stcg(idx_out + pos, idx[rd]);
-                            __stcg(keys_out + pos, key[rd]);
-                        }
-                    }
-                    if (!last) {
-                        // count the next digit per destination tile.  High digits are nearly constant over the
-                        // selection, so a warp sends one atomic per distinct counter instead of one per entry.
-                        const uint32_t nd = ((kmax - key[rd]) >> (shift + kSortBits)) & (kSortBins - 1);
-                        const uint32_t peers = match_digit(nd, live);
-                        const int leader = live ? __ffs(peers) - 1 : lane;
-                        const uint32_t t = pos >> tshift;
-                        const bool with_leader = t == __shfl_sync(0xFFFFFFFFu, t, leader);  // same destination tile as the leader
-                        const uint32_t same = __ballot_sync(0xFFFFFFFFu, live && with_leader);
-                        if (live) {
-                            if (lane == leader) atomicAdd(&cnt_next[static_cast<size_t>(t) * kSortBins + nd], static_cast<uint32_t>(__popc(peers & same)));
-                            else if (!with_leader) atomicAdd(&cnt_next[static_cast<size_t>(t) * kSortBins + nd], 1u);
+                            __stcg(pairs_out + pos, make_uint2(key[rd], static_cast<uint32_t>(idx[rd])));
                         }
                     }
                 }
             }
-            __syncthreads();
         }
         if (!last && !grid_sync<CLUSTER>(status, epoch)) return;
     }
