@@ -177,23 +177,53 @@ __device__ __forceinline__ void blank_slot(uint4& q, int e) {
 
 // The loss from the sum over the OTHER classes.  With M = max_{j != y} x_j, P = fl(M L) and
 // S = sum_{j != y} 2^(x_j L - P) (= 2^D sum_{j != y} exp(x_j - M), D = M L - P; S = 0 if there is no other class):
-//   x_y >= M:  l = log1p(sum_{j != y} exp(x_j - x_y)) = log1p(S 2^(P - x_y L))            (one fused multiply-add)
+//   x_y >= M:  l = log1p(u),  u = sum_{j != y} exp(x_j - x_y) = S 2^(P - x_y L)            (one fused multiply-add)
 //   x_y <  M:  l = (M - x_y) + log(sum_j exp(x_j - M)) = (M - x_y) + log((S + 2^(x_y L - P)) 2^-D)
 // Only sums of positive terms: nothing cancels, so a loss of 1e-9 is as accurate as a loss of 10, in one pass and
 // without a comparison per element (a small loss means that the true class dominates, so it is the true class, not
 // the maximum, that has to stay out of the sum).
+// Both forms are evaluated without a branch and one is selected: log1p(u) as its series up to u^6 below 1/8
+// (truncation 5e-7 relative) and as lg2(1 + u) ln 2 above (lg2.approx: 2^-22 absolute on a result above 0.11);
+// the second form's loss is above ln 2, where the same absolute error is 3e-7 relative.
+__device__ __forceinline__ float lg2(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ float loss_without_true_class(float M, float P, float S, float xy) {
-    if (xy >= M) return log1pf(S * ex2(fmaf(-xy, kLog2e, P)));
+    constexpr float kLn2 = 0.6931471805599453f;
+    const float u = S * ex2(fmaf(-xy, kLog2e, P));
+    float series = fmaf(u, -1.0f / 6.0f, 0.2f);
+    series = fmaf(u, series, -0.25f);
+    series = fmaf(u, series, 1.0f / 3.0f);
+    series = fmaf(u, series, -0.5f);
+    series = fmaf(u, series, 1.0f);
+    const float confident = u < 0.125f ? u * series : lg2(1.0f + u) * kLn2;
     const float D = fmaf(M, kLog2e, -P);
-    return (M - xy) + logf((S + ex2(fmaf(xy, kLog2e, -P))) * ex2(-D));
+    const float other = (M - xy) + (lg2(S + ex2(fmaf(xy, kLog2e, -P))) - D) * kLn2;
+    return xy >= M ? confident : other;
+}
+
+constexpr int kTinyThreads = 256;
+constexpr int kTinyMaxC = 32;
+constexpr int kTinyStages = 3;
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst))),
+                 "l"(gsrc)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
 }
 
 // ---------------------------------------------------------------------------
-// Tiny rows: a CTA stages 256 consecutive rows (contiguous in memory) into
-// shared memory with coalesced element loads; each thread then owns one row.
+// Tiny rows with a pool base that is not 16-byte aligned: a CTA stages 256
+// consecutive rows (contiguous in memory) into shared memory with coalesced
+// element loads; each thread then owns one row.
 // ---------------------------------------------------------------------------
-constexpr int kTinyThreads = 256;
-constexpr int kTinyMaxC = 32;
 
 template <typename T>
 __global__ void __launch_bounds__(kTinyThreads)
@@ -367,17 +397,6 @@ __device__ __forceinline__ void chunk_sum_exp(const typename ChunkWord<CB>::type
     }
 }
 
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst))),
-                 "l"(gsrc)
-                 : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int PENDING>
-__device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
-}
-
 // Tiles flow through a ring of kGroupStages buffers filled by asynchronous 16-byte copies (global -> shared, past
 // the registers), one tile ahead of the one being reduced, so every CTA always has loads in flight; two stages
 // rather than three leave room for a third CTA per SM, which is worth more (measured).
@@ -528,6 +547,180 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
         }
         __syncthreads();  // the stage may be refilled
         y = y_next;
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+    h.flush();
+}
+
+// ---------------------------------------------------------------------------
+// Short rows (up to kLaneMaxRowBytes), pool base 16-byte aligned: a WARP takes 32 consecutive rows (one
+// contiguous, 16-byte aligned byte range), brings them into its own ring of shared-memory stages with 16-byte
+// asynchronous copies, one or two blocks of rows ahead of the one being scored, and every LANE scores one row.
+// Nothing in the loop synchronises more than a warp, and the per-row work (label, reductions, the logarithm) is
+// done once per lane instead of once per group of lanes.  Rows that are whole 16-byte chunks are laid out at an
+// odd chunk pitch; other rows are copied flat and read in units of the largest power of two (8, 4 or 2 bytes) that
+// divides the row length, so that the lanes' strides are odd multiples of the unit: no bank conflicts either way.
+// CMAX > 0 (rows of at most 32 elements): the row is read once into CMAX registers (slots past C hold -inf).
+// CMAX == 0: two passes over the row in shared memory (maximum, then the sum), in units of CB bytes.
+// A row's sum runs over its elements in an order that depends on C only, so copies of a row score the same bits
+// wherever they sit.
+// ---------------------------------------------------------------------------
+constexpr int kLaneThreads = 128;
+constexpr int kLaneMaxRowBytes = 416;
+
+template <typename T, int CMAX, int CB, int STAGES>
+__global__ void __launch_bounds__(CMAX > 0 ? kTinyThreads : kLaneThreads)
+score_lane_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
+                       int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0,
+                       int stage_bytes) {
+    constexpr bool PADDED = CB == 16;
+    constexpr int kWarpsPerCta = (CMAX > 0 ? kTinyThreads : kLaneThreads) / 32;
+    extern __shared__ __align__(16) unsigned char lane_smem[];
+    uint32_t* hist_s = reinterpret_cast<uint32_t*>(lane_smem);
+    Hist0 h{hist_s, hist0};
+    h.clear();
+    __syncthreads();
+    constexpr int ES = static_cast<int>(sizeof(T));
+    constexpr int EPC = 16 / ES;  // elements per 16-byte chunk
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned char* ring = lane_smem + kSelBins * sizeof(uint32_t) + static_cast<size_t>(warp) * STAGES * stage_bytes;
+    const int row_bytes = C * ES;
+    const int rc = PADDED ? row_bytes >> 4 : 1;  // chunks per row
+    const int pitch = rc | 1;                     // odd: the eight lanes of a quarter-warp read eight different bank groups
+    const int64_t blocks = (rows + 31) >> 5;
+    const int64_t gw = static_cast<int64_t>(blockIdx.x) * kWarpsPerCta + warp;
+    const int64_t nw = static_cast<int64_t>(gridDim.x) * kWarpsPerCta;
+    const int64_t mine = blocks > gw ? (blocks - gw + nw - 1) / nw : 0;
+    const float inv_rc = 1.0f / static_cast<float>(rc);
+
+    auto place = [&](int v) -> int {  // chunk v of a block of rows -> its chunk slot in the stage
+        if constexpr (!PADDED) return v;
+        const int r = __float2int_rz((static_cast<float>(v) + 0.5f) * inv_rc);  // v / rc, exact for v < 2^20
+        return r * pitch + (v - r * rc);
+    };
+    auto issue = [&](int64_t i) -> int64_t {  // requests this warp's i-th block of rows; returns this lane's label
+        int64_t y = ignore_index;
+        if (i < mine) {
+            const int64_t row0 = (gw + i * nw) << 5;
+            const int nrows = rows - row0 < 32 ? static_cast<int>(rows - row0) : 32;
+            const unsigned char* src = reinterpret_cast<const unsigned char*>(logits) + row0 * row_bytes;
+            unsigned char* dst = ring + (i % STAGES) * stage_bytes;
+            const int bytes = nrows * row_bytes, nvec = bytes >> 4;
+            for (int v = lane; v < nvec; v += 32) cp_async16(dst + place(v) * 16, src + v * 16);
+            // a last, partial chunk (only at the very end of the pool) is copied element by element
+            for (int e = (nvec << 4) / ES + lane; e < bytes / ES; e += 32) {
+                const int byte = e * ES;
+                *reinterpret_cast<T*>(dst + place(byte >> 4) * 16 + (byte & 15)) = reinterpret_cast<const T*>(src)[e];
+            }
+            if (lane < nrows) y = labels[row0 + lane];
+        }
+        cp_async_commit();  // one group per slot, also when it is empty: the wait below counts groups
+        return y;
+    };
+
+    int64_t yq[STAGES - 1];
+#pragma unroll
+    for (int i = 0; i < STAGES - 1; ++i) yq[i] = issue(i);
+    for (int64_t i = 0; i < mine; ++i) {
+        const int64_t y_new = issue(i + STAGES - 1);
+        const int64_t y = yq[0];
+#pragma unroll
+        for (int q = 0; q + 1 < STAGES - 1; ++q) yq[q] = yq[q + 1];
+        yq[STAGES - 2] = y_new;
+        cp_async_wait<STAGES - 1>();
+        __syncwarp();  // every lane's copies of block i have landed
+        const int64_t row0 = (gw + i * nw) << 5;
+        const bool valid = row0 + lane < rows;
+        unsigned char* buf = ring + (i % STAGES) * stage_bytes;
+        const int cls = valid ? label_class(y, C, ignore_index) : 1;
+        T* rowe = reinterpret_cast<T*>(buf + (PADDED ? lane * pitch * 16 : lane * row_bytes));
+        // the true class stays out of the sum (see loss_without_true_class): its slot is read, then blanked
+        float xy = 0.f;
+        if (cls == 0) {
+            xy = Elem<T>::widen(rowe[static_cast<int>(y)]);
+            rowe[static_cast<int>(y)] = Elem<T>::neg_inf_elem();
+        }
+        float m = -1e30f, s = 0.f;
+        if constexpr (CMAX > 0) {
+            float x[CMAX];
+            if constexpr (PADDED) {
+                constexpr int kCh = CMAX / EPC;
+                const uint4* rowv = reinterpret_cast<const uint4*>(rowe);
+#pragma unroll
+                for (int c = 0; c < kCh; ++c) {
+                    if (c < rc) {
+                        const uint4 q = rowv[c];
+                        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            if constexpr (ES == 4) {
+                                x[c * 4 + e] = __uint_as_float(w[e]);
+                            } else {
+                                x[c * 8 + 2 * e] = __uint_as_float(w[e] << 16);
+                                x[c * 8 + 2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < EPC; ++e) x[c * EPC + e] = neg_inf();
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < CMAX; ++j) x[j] = j < C ? Elem<T>::widen(rowe[j]) : neg_inf();
+            }
+            __syncwarp();  // the stage may be refilled by the next issue
+#pragma unroll
+            for (int j = 0; j < CMAX; ++j) m = fmaxf(m, x[j]);
+            const float P = m * kLog2e;
+            const F2 l2e = pack2(kLog2e, kLog2e), nml = pack2(-P, -P);
+            F2 acc = pack2(0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < CMAX; j += 2) pair_sum_exp(x[j], x[j + 1], l2e, nml, acc);
+            float s0, s1;
+            unpack2(acc, s0, s1);
+            s = s0 + s1;
+        } else if constexpr (CB * 2 > ES * 2 && CB >= 2 * ES) {
+            // units of at least two elements: maximum on whole units (bf16: packed pairs), two-wide sums
+            using Word = typename ChunkWord<CB>::type;
+            const Word* xv = reinterpret_cast<const Word*>(rowe);
+            const int nch = cls == 0 ? (PADDED ? rc : row_bytes / CB) : 0;
+            ChunkMax<T> cm;
+#pragma unroll 4
+            for (int c = 0; c < nch; ++c) cm.template add<CB>(xv[c]);
+            m = fmaxf(m, cm.get());
+            const float P = m * kLog2e;
+            const F2 l2e = pack2(kLog2e, kLog2e), nml = pack2(-P, -P);
+            F2 a0 = pack2(0.f, 0.f), a1 = pack2(0.f, 0.f);
+#pragma unroll 4
+            for (int c = 0; c < nch; ++c) chunk_sum_exp<T, CB>(xv[c], l2e, nml, a0, a1);
+            float t0, t1, t2, t3;
+            unpack2(a0, t0, t1);
+            unpack2(a1, t2, t3);
+            s = (t0 + t1) + (t2 + t3);
+            __syncwarp();
+        } else {
+            // single elements (rows of an odd number of elements)
+            const int n = cls == 0 ? C : 0;
+#pragma unroll 4
+            for (int j = 0; j < n; ++j) m = fmaxf(m, Elem<T>::widen(rowe[j]));
+            const float P = m * kLog2e;
+#pragma unroll 4
+            for (int j = 0; j < n; ++j) s += ex2(fmaf(Elem<T>::widen(rowe[j]), kLog2e, -P));
+            __syncwarp();
+        }
+        float loss = 0.f;
+        if (cls == 2) {
+            loss = __uint_as_float(0x7FC00000u);
+            atomicAdd(&status->bad_labels, 1);
+        } else if (cls == 0) {
+            loss = loss_without_true_class(m, m * kLog2e, s, xy);
+        }
+        if (valid) {
+            row_loss[row0 + lane] = loss;
+            h.add(loss);
+        }
     }
     cp_async_wait<0>();
     __syncthreads();
@@ -774,6 +967,49 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
     const int sms = sm_count();
     const int64_t max_ctas = test_geometry().max_ctas;
     const int64_t row_bytes = C * static_cast<int64_t>(sizeof(T));
+    const bool base16 = (reinterpret_cast<uintptr_t>(logits) & 15) == 0;
+    if (base16 && (C <= kTinyMaxC || row_bytes <= kLaneMaxRowBytes)) {
+        // one lane per row: the access unit is the largest power of two (at most 16 bytes) that divides the row
+        cudaError_t err = cudaSuccess;
+        const int cb = row_bytes % 16 == 0 ? 16 : row_bytes % 8 == 0 ? 8 : row_bytes % 4 == 0 ? 4 : 2;
+        auto go = [&](auto kernel, int threads, int stages) {
+            const int64_t rc = row_bytes / 16;
+            const int stage_bytes = static_cast<int>(cb == 16 ? 32 * (rc | 1) * 16 : (32 * row_bytes + 15) / 16 * 16);
+            const size_t smem = kSelBins * sizeof(uint32_t) + static_cast<size_t>(threads / 32) * stages * stage_bytes;
+            err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynSmem));
+            if (err != cudaSuccess) return;
+            const int64_t want = ((rows + 31) / 32 + threads / 32 - 1) / (threads / 32);
+            const int grid = static_cast<int>(std::min({want, static_cast<int64_t>(sms) * blocks_per_sm(kernel, threads, smem), max_ctas}));
+            kernel<<<grid, threads, smem, s>>>(logits, labels, rows, static_cast<int>(C), ignore_index, row_loss, status,
+                                               hist0, stage_bytes);
+            err = cudaGetLastError();
+        };
+        if (C <= kTinyMaxC) {
+            auto by_len = [&](auto cb_tag) {
+                constexpr int CBT = decltype(cb_tag)::value;  // 16: rows are whole chunks; 0: anything else
+                constexpr bool f32 = sizeof(T) == 4;
+                if (C <= 4) go(score_lane_rows_kernel<T, 4, f32 ? CBT : 0, kTinyStages>, kTinyThreads, kTinyStages);
+                else if (C <= 8) go(score_lane_rows_kernel<T, 8, CBT, kTinyStages>, kTinyThreads, kTinyStages);
+                else if (C <= 12) go(score_lane_rows_kernel<T, 12, f32 ? CBT : 0, kTinyStages>, kTinyThreads, kTinyStages);
+                else if (C <= 16) go(score_lane_rows_kernel<T, 16, CBT, kTinyStages>, kTinyThreads, kTinyStages);
+                else if (C <= 24) go(score_lane_rows_kernel<T, 24, CBT, kTinyStages>, kTinyThreads, kTinyStages);
+                else go(score_lane_rows_kernel<T, 32, CBT, kTinyStages>, kTinyThreads, kTinyStages);
+            };
+            if (cb == 16) by_len(std::integral_constant<int, 16>{});
+            else by_len(std::integral_constant<int, 0>{});
+            return err;
+        }
+        auto by_unit = [&](auto stages_tag) {
+            constexpr int ST = decltype(stages_tag)::value;
+            if (cb == 16) go(score_lane_rows_kernel<T, 0, 16, ST>, kLaneThreads, ST);
+            else if (cb == 8) go(score_lane_rows_kernel<T, 0, 8, ST>, kLaneThreads, ST);
+            else if (cb == 4) go(score_lane_rows_kernel<T, 0, 4, ST>, kLaneThreads, ST);
+            else go(score_lane_rows_kernel<T, 0, 2, ST>, kLaneThreads, ST);
+        };
+        if (32 * row_bytes <= 6144) by_unit(std::integral_constant<int, 3>{});
+        else by_unit(std::integral_constant<int, 2>{});
+        return err;
+    }
     if (C <= kTinyMaxC) {
         const int64_t tiles = (rows + kTinyThreads - 1) / kTinyThreads;
         const int grid = static_cast<int>(std::min({tiles, static_cast<int64_t>(sms) * 8, max_ctas}));

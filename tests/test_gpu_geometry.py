@@ -68,7 +68,8 @@ def pads_intact(buf, nbytes, fill=0x5A):
 
 
 # one shape per scorer kernel, each several tiles with a ragged tail
-SCORER_SHAPES = [(20_011, 1, 10, "f32"), (9_001, 1, 32, "bf16"), (30_011, 1, 100, "f32"), (20_003, 1, 100, "bf16"),
+SCORER_SHAPES = [(20_011, 1, 10, "f32"), (9_001, 1, 32, "bf16"), (30_011, 1, 100, "f32"), (20_003, 1, 100, "bf16"), (7_001, 1, 101, "bf16"),
+                 (6_007, 1, 103, "f32"),
                  (5_003, 1, 200, "f32"), (4_001, 1, 1000, "bf16"), (3_001, 1, 5000, "f32"), (257, 4, 30_522, "bf16"),
                  (37, 1, 70_001, "f32")]
 

@@ -50,7 +50,10 @@ def random_pool(seed, N, T, C, dtype, sigma=2.0, bump=1.0, mask_p=0.0):
 SCORE_SHAPES = [
     # N, T, C, dtype            path
     (1, 1, 1, "f32"), (33, 1, 2, "f32"), (1000, 1, 3, "f32"), (777, 1, 7, "bf16"), (5000, 1, 10, "f32"),
-    (300, 1, 32, "bf16"),                                                        # tiny rows
+    (300, 1, 32, "bf16"), (2000, 1, 4, "f32"), (1111, 1, 5, "bf16"), (999, 1, 12, "f32"), (640, 1, 16, "bf16"), (1500, 1, 20, "f32"),
+    (901, 1, 24, "bf16"), (1300, 1, 28, "f32"), (77, 1, 31, "f32"),             # rows of at most 32 elements: one lane per row, in registers
+    (500, 1, 33, "bf16"), (700, 1, 101, "bf16"), (400, 1, 104, "f32"), (300, 1, 105, "f32"), (1200, 1, 50, "bf16"), (900, 1, 52, "f32"),
+    (2500, 1, 208, "bf16"), (1000, 1, 103, "f32"),                              # one lane per row out of shared memory, units of 16/8/4/2 bytes
     (31, 1, 33, "f32"), (2049, 1, 100, "f32"), (513, 1, 100, "bf16"),
     (1000, 1, 36, "f32"), (333, 2, 40, "bf16"), (4099, 1, 64, "f32"), (777, 1, 102, "f32"), (650, 1, 128, "bf16"),
     (129, 3, 128, "f32"), (1031, 1, 132, "f32"), (500, 1, 200, "f32"), (97, 2, 201, "f32"), (420, 1, 256, "f32"),
