@@ -47,12 +47,12 @@ def measured_peak():
 # algorithmic bytes
 # --------------------------------------------------------------------------- #
 def score_topk_bytes(cfg, labels: np.ndarray) -> int:
-    """Logits of the unmasked rows + every label + the loss table in and out of the selector + k indices and values."""
+    """Scorer: logits + loss of every unmasked row, every label; selector: the loss table read once, k indices and values."""
     es = 4 if cfg.dtype == "f32" else 2
     unmasked = int((labels != wl.IGNORE_INDEX).sum())
     rows = labels.size
     b = unmasked * (cfg.C * es + 4) + rows * 8
-    b += 4 * cfg.N + 4 * cfg.N + 8 * cfg.k
+    b += 4 * cfg.N + 8 * cfg.k
     return b
 
 
@@ -195,7 +195,7 @@ def run_reference(args, cfg):
         "impl": "reference", "metric": "score+top-k samples/s", "value": value, "unit": "samples/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(cfg, "host memory; CPU oracle"),
+        "config": workload_config(cfg), "inputs": "host memory; CPU oracle",
         "aggregation": {"value": 4 * d * (cfg.P + 1) * args.steps / ta / 1e9, "unit": "GB/s"},
         "cpu_baseline": {"value": value, "unit": "samples/s", "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "samples/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -224,22 +224,22 @@ def job_throughput(world: int, units_per_rank: float, steps: int, ms: float) -> 
     return world * units_per_rank * steps / (ms * 1e-3)
 
 
-# DRAM traffic per launch (dram__bytes_read + dram__bytes_write) from the ncu captures summarised under
-# profiles/, taken on a scaled-down case and scaled to a full launch by the units processed.  Only for the
-# kernels and workloads that were captured; None elsewhere (and to be reset when a kernel changes).
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernels, from ncu captures of
+# scaled-down cases (128 of config 4's 1,024 sequences; 16,000,000 of its 109,482,240 parameters per replica), scaled
+# to a full launch by the units processed.  Valid only for the kernels as captured: reset to None whenever
+# score_stream_rows_kernel or aggregate_vec4_kernel changes, until the counters have been taken again.
 NCU_TRAFFIC_BYTES = {
-    ("score", 4): 7.28e9,      # profiles/score_stream_rows_bf16_cfg4.md: 909.4 MB for 128 of 1024 sequences
-    ("aggregate", 4): 4.70e9,  # profiles/aggregate_vec4_cfg4.md: 687.0 MB for 16,000,000 of 109,482,240 parameters
+    ("score", 4): 7.27e9,      # 908.5 MB for 128 of 1,024 sequences
+    ("aggregate", 4): 4.77e9,  # 697.8 MB for 16,000,000 of 109,482,240 parameters
 }
 
 
-def workload_config(cfg, residency: str):
+def workload_config(cfg):
     return {
         "workload": f"config {cfg.cfg_id} ({cfg.name}-scale round): pool {cfg.N} x {cfg.T} x {cfg.C} {cfg.dtype} logits, "
                     f"k={cfg.k}; {cfg.P} replicas x {cfg.D} fp32 parameters",
         "N": cfg.N, "T": cfg.T, "C": cfg.C, "k": cfg.k, "P": cfg.P, "D": cfg.D, "order": "loss_desc",
         "l2": "inputs larger than L2 (no flush needed)" if cfg.logit_bytes > (1 << 28) else "L2 flushed between steps",
-        "inputs": residency,
     }
 
 
@@ -329,18 +329,30 @@ def run_gpu(args, cfg):
     # pools that fit in L2 were timed cold (flushed before every step); also give the warm figure
     warm = None
     if flush is not None:
-        w_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(20)]
+        # the two calls captured once each into CUDA graphs and replayed: the device's time for a step whose inputs
+        # may sit in L2, without the host's enqueue cost (which bounds eagerly launched steps shorter than ~60 us)
+        side = torch.cuda.Stream()
+        graphs = []
+        with torch.cuda.stream(side):
+            for call in (lambda: lsgd.score_topk(d_logits, d_labels, cfg.k, lsgd.ORDER_LOSS_DESC, losses=losses, out_idx=idx,
+                                                 out_vals=vals, ws=ws),
+                         lambda: lsgd.aggregate(d_reps, weights, out=out)):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    call()
+                graphs.append(g)
+        torch.cuda.synchronize()
+        w_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(23)]
         for e in w_ev:
             e[0].record()
-            lsgd.score_topk(d_logits, d_labels, cfg.k, lsgd.ORDER_LOSS_DESC, losses=losses, out_idx=idx, out_vals=vals, ws=ws)
+            graphs[0].replay()
             e[1].record()
-            lsgd.aggregate(d_reps, weights, out=out)
+            graphs[1].replay()
             e[2].record()
         torch.cuda.synchronize()
-        warm = {"score_topk_ms": float(np.median([e[0].elapsed_time(e[1]) for e in w_ev])),
-                "aggregate_ms": float(np.median([e[1].elapsed_time(e[2]) for e in w_ev])),
-                "note": "same step without the L2 flush (inputs may be L2-resident); median of 20; with nothing between the "
-                        "steps the host's enqueue rate, not the device, bounds steps shorter than about 60 us"}
+        warm = {"score_topk_ms": float(np.median([e[0].elapsed_time(e[1]) for e in w_ev[3:]])),
+                "aggregate_ms": float(np.median([e[1].elapsed_time(e[2]) for e in w_ev[3:]])),
+                "note": "the same two calls replayed from CUDA graphs without the L2 flush (inputs may be L2-resident); median of 20"}
 
     # ---- end to end: inputs from pinned host memory, results back to the host, every step
     e2e_steps = max(1, min(args.steps, 5 if cfg.logit_bytes > (1 << 30) else 20))
@@ -440,7 +452,7 @@ def run_gpu(args, cfg):
             "metric": "score+top-k samples/s", "value": job_throughput(world, cfg.N, args.steps, st_sum), "unit": "samples/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(cfg, "resident in HBM"),
+            "config": workload_config(cfg), "inputs": "resident in HBM",
             "score_topk": {"ms": st_sum / args.steps, "ms_best": float(st_ms.min()), "gbs": st_gbs,
                            "frac_of_measured_hbm": st_gbs / peak, "frac_of_nominal_8tbs": st_gbs / NOMINAL_HBM_GBS,
                            "algorithmic_bytes": st_bytes, "bad_labels": bad},
@@ -512,6 +524,9 @@ def run_scorer_sweep(args):
     # in which the loss keeps its relative accuracy only through the max-excluded sum
     shapes += [(r, C, dt, 14.0) for r, C, dt in SWEEP_SHAPES if (C, dt) in ((100, "f32"), (1000, "f32"), (8000, "f32"),
                                                                            (300, "bf16"), (4000, "bf16"), (30522, "bf16"))]
+    if args.sweep_filter:  # "C:dtype[:rows]": that row shape alone (profiling runs), optionally with fewer rows
+        f = args.sweep_filter.split(":")
+        shapes = [(int(f[2]) if len(f) > 2 else r, C, dt, b) for r, C, dt, b in shapes if C == int(f[0]) and dt == f[1] and b == 0.0]
     for rows, C, dt, bump in shapes:
         tdt = torch.float32 if dt == "f32" else torch.bfloat16
         g = torch.Generator(device="cuda").manual_seed(MASTER_SWEEP_SEED + C)
@@ -547,6 +562,32 @@ def run_scorer_sweep(args):
 MASTER_SWEEP_SEED = 20250808
 
 
+def spawn_ranks(n: int, argv, timeout_s: float | None = None) -> int:
+    """Starts `n` copies of the command `argv`, one per GPU of this node, with the environment a torchrun launch
+    would give them (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR = 127.0.0.1, a free MASTER_PORT), and waits for them.
+    The children share this process's stdout (rank 0 prints the JSON line).  Returns the worst exit code.
+    The ranks run independent replicas of the round; they only meet for barriers and the max over their timings."""
+    import socket
+    import subprocess
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen(list(argv), env=env))
+    worst = 0
+    for pr in procs:
+        try:
+            rc = pr.wait(timeout=timeout_s)
+        except subprocess.TimeoutExpired:
+            pr.kill()
+            rc = 124
+        worst = max(worst, abs(rc))
+    return worst
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -557,6 +598,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep-scorer", action="store_true",
                     help="instead of the round: time lsgd_score_losses alone over a range of row lengths (1 GPU)")
+    ap.add_argument("--sweep-filter", default="", help="with --sweep-scorer: only the row shape C:dtype[:rows]")
     ap.add_argument("--no-round", action="store_true", help="skip the lsgd_aggregate_round legs (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--n-samples", type=int, default=0, help="profiling: shrink the pool to this many samples")
@@ -566,6 +608,9 @@ def main():
     if args.n_samples or args.d_params:
         n = args.n_samples or cfg.N
         cfg = wl.scaled(cfg, name=cfg.name + "-scaled", N=n, k=max(1, cfg.k * n // cfg.N), D=args.d_params or cfg.D)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference" and not args.sweep_scorer:
+        # started plainly with --gpus N: become the launcher of N ranks (under torchrun the environment is already set)
+        sys.exit(spawn_ranks(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:]))
     if args.sweep_scorer:
         args.steps = min(args.steps, 20)
         run_scorer_sweep(args)
