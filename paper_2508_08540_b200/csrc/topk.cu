@@ -21,13 +21,16 @@
 //      if all selected keys are equal); stability turns the index-ascending input
 //      order into the required tie-break.  A pass is two phases: rank every tile
 //      by the digit (which gives the tile's digit counts), then scatter.
-// The kernel runs either as ONE thread-block cluster (pools of up to 65,536
-// entries: the barrier is the cluster's hardware barrier) or as a cooperative
-// launch with one block per multiprocessor (all blocks resident by construction;
-// the barrier is an arrival counter in the status block, polled with a limit: if
-// it ever ran out, the block would set the status block's timeout word and
-// return, and the other blocks would follow).
+// Pools of up to 65,536 entries run as ONE thread-block cluster that keeps all it
+// exchanges in distributed shared memory (topk_cluster_kernel: the barrier is the
+// cluster's hardware barrier); larger pools as a cooperative launch with one
+// block per multiprocessor that exchanges through the workspace (all blocks
+// resident by construction; the barrier is an arrival counter in the status
+// block, polled with a limit: if it ever ran out, the block would set the status
+// block's timeout word and return, and the other blocks would follow).
 // Pools of at most kSmallN entries are sorted whole by a single block instead.
+#include <cooperative_groups.h>
+
 #include <algorithm>
 
 #include "lsgd_internal.cuh"
@@ -120,39 +123,33 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
     return v;
 }
 
-// Barrier over all blocks of the kernel, with the other blocks' global writes visible afterwards (read them with
-// __ldcg).  CLUSTER: the grid is one cluster, the barrier is the cluster's.  Otherwise (cooperative launch): an
-// arrival counter that only grows; barrier number e is passed once e * gridDim.x arrivals are in.  Returns false
-// if the wait ran out (or another block's did): the caller returns at once.
-template <bool CLUSTER>
+// Barrier over all blocks of a cooperatively launched kernel, with the other blocks' global writes visible
+// afterwards (read them with __ldcg): an arrival counter that only grows; barrier number e is passed once
+// e * gridDim.x arrivals are in.  Returns false if the wait ran out (or another block's did): the caller returns
+// at once.
 __device__ __forceinline__ bool grid_sync(StatusBlock* st, uint32_t& epoch) {
-    if constexpr (CLUSTER) {
-        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-        return true;
-    } else {
-        __shared__ int ok_s;
-        ++epoch;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            const uint32_t target = epoch * gridDim.x;
-            __threadfence();
-            atomicAdd(&st->grid_arrivals, 1u);
-            int ok = 1;
-            uint32_t polls = 0;
-            while (ld_acquire(&st->grid_arrivals) < target) {
-                if (++polls > kMaxPolls || ((polls & 63u) == 0 && *reinterpret_cast<volatile int32_t*>(&st->timeout) != 0)) {
-                    ok = 0;
-                    break;
-                }
-                __nanosleep(32);
+    __shared__ int ok_s;
+    ++epoch;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t target = epoch * gridDim.x;
+        __threadfence();
+        atomicAdd(&st->grid_arrivals, 1u);
+        int ok = 1;
+        uint32_t polls = 0;
+        while (ld_acquire(&st->grid_arrivals) < target) {
+            if (++polls > kMaxPolls || ((polls & 63u) == 0 && *reinterpret_cast<volatile int32_t*>(&st->timeout) != 0)) {
+                ok = 0;
+                break;
             }
-            if (!ok) atomicExch(&st->timeout, 1);
-            __threadfence();
-            ok_s = ok;
+            __nanosleep(32);
         }
-        __syncthreads();
-        return ok_s != 0;
+        if (!ok) atomicExch(&st->timeout, 1);
+        __threadfence();
+        ok_s = ok;
     }
+    __syncthreads();
+    return ok_s != 0;
 }
 
 // Block-wide exclusive scan of one value per thread.  `warp_tot` holds kWarps + 1 words; the block total is left
@@ -185,12 +182,13 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* w
 
 // Walks a finished histogram (global memory) from its highest bin down and finds the bin that holds the `want`-th
 // entry (1-based).  On return (all threads): bin, and `want` reduced by the entries in the bins above it.
+template <bool GLOBAL = true>
 __device__ void find_bin(const uint32_t* hist, int nbins, uint32_t& want, uint32_t& bin, uint32_t* warp_tot, uint32_t* result) {
     // thread t owns bins nbins - 1 - 2 t and nbins - 2 - 2 t (or the single bin nbins - 1 - t), highest first
     const bool two = nbins == 2 * kThreads;
     const int b0 = two ? nbins - 1 - 2 * static_cast<int>(threadIdx.x) : nbins - 1 - static_cast<int>(threadIdx.x);
-    const uint32_t c0 = __ldcg(hist + b0);
-    const uint32_t c1 = two ? __ldcg(hist + b0 - 1) : 0u;
+    const uint32_t c0 = GLOBAL ? __ldcg(hist + b0) : hist[b0];
+    const uint32_t c1 = !two ? 0u : GLOBAL ? __ldcg(hist + b0 - 1) : hist[b0 - 1];
     const uint32_t before = block_exclusive_scan(c0 + c1, warp_tot);
     if (before < want && want <= before + c0 + c1) {
         const bool first = want <= before + c0;
@@ -241,7 +239,7 @@ __device__ __forceinline__ uint32_t match_digit(uint32_t d, bool live) {
 }
 
 // E: keys per thread of a selection tile (tiles of 1024 E entries; block b takes tiles b, b + gridDim.x, ...).
-template <int E, bool CLUSTER>
+template <int E>
 __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_constant__ SelectParams p) {
     extern __shared__ __align__(16) uint32_t dyn_smem[];  // selection: hist_s[kSelBins]; sort: counters[kWarps][kCounterPitch]
     __shared__ uint32_t warp_tot[kWarps + 1];
@@ -289,14 +287,9 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
 #pragma unroll
             for (int i = 0; i < E; ++i) {
                 const bool in = key[i] != 0u && (key[i] & mask) == prefix;
-                if (pass == 0) {
-                    // every key counts and losses crowd into a few bins: one atomic per distinct digit and warp
-                    const uint32_t d = in ? digit_of(key[i], 0) : 0xFFFFFFFFu;
-                    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, d);
-                    if (in && lane == __ffs(peers) - 1) atomicAdd(&hist_s[d], __popc(peers));
-                } else if (in) {
-                    atomicAdd(&hist_s[digit_of(key[i], pass)], 1u);
-                }
+                // plain shared-memory atomics: measured faster than warp-aggregated ones (match.any) for crowded, uniform and
+                // all-equal keys alike
+                if (in) atomicAdd(&hist_s[digit_of(key[i], pass)], 1u);
             }
         });
         __syncthreads();
@@ -306,7 +299,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
             if (c) atomicAdd(&gh[i], c);
             hist_s[i] = 0;
         }
-        if (!grid_sync<CLUSTER>(status, epoch)) return;
+        if (!grid_sync(status, epoch)) return;
         uint32_t bin;
         find_bin(gh, pass == 2 ? 1024 : kSelBins, want, bin, warp_tot, result);
         prefix |= pass == 0 ? bin << 21 : pass == 1 ? bin << 10 : bin;
@@ -340,7 +333,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
         }
         __syncthreads();
     });
-    if (!grid_sync<CLUSTER>(status, epoch)) return;
+    if (!grid_sync(status, epoch)) return;
 
     // ---- 3. ordered compaction ----
     // The sort key of a selected entry is u = kmax - key (0 for the largest loss); `passes` 9-bit digits cover its range.
@@ -409,7 +402,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
         __syncthreads();
     });
     if (direct) return;
-    if (!grid_sync<CLUSTER>(status, epoch)) return;
+    if (!grid_sync(status, epoch)) return;
 
     // ---- 4. stable LSD sort of the k pairs on u = kmax - key, ascending, 9 bits per pass ----
     // A pass has two halves with a barrier between them: every tile ranks its entries by the pass's digit
@@ -486,7 +479,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
         } else {
             for (uint32_t tile = blockIdx.x; tile < St; tile += gridDim.x) rank_tile(tile, true);
         }
-        if (!grid_sync<CLUSTER>(status, epoch)) return;
+        if (!grid_sync(status, epoch)) return;
 
         for (uint32_t tile = blockIdx.x; tile < St; tile += gridDim.x) {
             if (!one_tile) {
@@ -563,7 +556,285 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
                 }
             }
         }
-        if (!last && !grid_sync<CLUSTER>(status, epoch)) return;
+        if (!last && !grid_sync(status, epoch)) return;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Pools of up to kMaxClusterBlocks x 8,192 entries: the same algorithm as ONE thread-block cluster, everything
+// that blocks exchange kept in (distributed) shared memory.  Block b owns entries [8192 b, 8192 b + 8192) of the
+// pool (in registers) and sort tile b.  Digit histograms are added into block 0's shared memory and read from
+// there by every block; per-block counts, the sort's digit counts and the (key, index) pairs themselves are
+// written straight into the destination block's shared memory.  The barrier is the cluster's hardware barrier.
+// ---------------------------------------------------------------------------
+namespace cg = cooperative_groups;
+
+constexpr int kClE = 8;
+constexpr int kClTile = kThreads * kClE;
+constexpr size_t kClCountersBytes = sizeof(uint32_t) * kWarps * kCounterPitch;
+constexpr size_t kClPairsBytes = sizeof(uint2) * 2 * kClTile;
+constexpr size_t kClMatBytes = sizeof(uint32_t) * kMaxClusterBlocks * kSortBins;
+constexpr size_t kClSmemBytes = kClCountersBytes + kClPairsBytes + kClMatBytes + sizeof(uint4) * kMaxClusterBlocks;
+static_assert(kClCountersBytes % 16 == 0, "the pair buffers start 16-byte aligned");
+static_assert(sizeof(uint32_t) * kSelPasses * kSelBins <= kClPairsBytes / 2, "the selection's histograms fit in the first pair buffer");
+
+__global__ void __launch_bounds__(kThreads, 1) topk_cluster_kernel(const __grid_constant__ SelectParams p) {
+    extern __shared__ __align__(16) unsigned char cl_smem[];
+    uint32_t* dyn = reinterpret_cast<uint32_t*>(cl_smem);                                   // hist_s, later counters
+    uint2* pairs = reinterpret_cast<uint2*>(cl_smem + kClCountersBytes);                     // [2][kClTile]
+    uint32_t* acc_hist = reinterpret_cast<uint32_t*>(pairs);                                 // block 0, selection only: [3][kSelBins]
+    uint32_t* mat = reinterpret_cast<uint32_t*>(cl_smem + kClCountersBytes + kClPairsBytes);  // [blocks][kSortBins]
+    uint4* cta_cnt = reinterpret_cast<uint4*>(cl_smem + kClCountersBytes + kClPairsBytes + kClMatBytes);
+    __shared__ uint32_t warp_tot[kWarps + 1];
+    __shared__ uint32_t result[2];
+    __shared__ uint32_t red[3];
+    __shared__ uint32_t digit_s[2];  // (bin, rank left) of the digit block 0 resolved last
+    __shared__ uint32_t base_s[kSortBins], tot_s[kSortBins], half_cnt[2][kSortBins];
+    cg::cluster_group cluster = cg::this_cluster();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t rank = blockIdx.x, nblocks = gridDim.x;
+    const float* __restrict__ losses = p.losses;
+    const int64_t N = p.N;
+    uint32_t* hist_s = dyn;
+
+    for (int i = tid; i < kSelBins; i += kThreads) hist_s[i] = 0;
+    for (int i = tid; i < kSelPasses * kSelBins; i += kThreads) acc_hist[i] = 0;
+    for (int i = tid; i < kMaxClusterBlocks * kSortBins; i += kThreads) mat[i] = 0;
+    if (tid < 3) red[tid] = 0;
+    cluster.sync();          // every block's accumulators are clear before anybody adds to them
+    grid_dependency_wait();  // the losses (and the scorer's histogram) are complete from here on
+
+    uint32_t key[kClE];
+    load_keys<kClE>(losses, N, static_cast<int64_t>(rank) * kClTile + static_cast<int64_t>(tid) * kClE, key);
+
+    // ---- 1. radix select ----
+    uint32_t prefix = 0, want = p.k;
+    if (p.hist0_ready) {
+        uint32_t bin;
+        find_bin(p.ws.hist, kSelBins, want, bin, warp_tot, result);
+        prefix = bin << 21;
+    }
+    for (int pass = p.hist0_ready ? 1 : 0; pass < kSelPasses; ++pass) {
+        const uint32_t mask = prefix_mask(pass);
+        __syncthreads();  // hist_s is zero
+#pragma unroll
+        for (int i = 0; i < kClE; ++i) {
+            const bool in = key[i] != 0u && (key[i] & mask) == prefix;
+            // plain shared-memory atomics: measured faster than warp-aggregated ones (match.any) for crowded, uniform and
+            // all-equal keys alike
+            if (in) atomicAdd(&hist_s[digit_of(key[i], pass)], 1u);
+        }
+        __syncthreads();
+        uint32_t* acc0 = cluster.map_shared_rank(acc_hist, 0) + pass * kSelBins;
+        for (int i = tid; i < kSelBins; i += kThreads) {
+            const uint32_t c = hist_s[i];
+            if (c) atomicAdd(acc0 + i, c);
+            hist_s[i] = 0;
+        }
+        cluster.sync();
+        // block 0 resolves the digit from its own shared memory and tells every block (reading 2,048 bins of
+        // another block's shared memory from every block took longer than this second barrier)
+        if (rank == 0) {
+            uint32_t bin;
+            find_bin<false>(acc_hist + pass * kSelBins, pass == 2 ? 1024 : kSelBins, want, bin, warp_tot, result);
+            if (tid < static_cast<int>(nblocks)) {
+                uint32_t* dst = cluster.map_shared_rank(digit_s, tid);
+                dst[0] = bin;
+                dst[1] = want;
+            }
+        }
+        cluster.sync();
+        const uint32_t bin = digit_s[0];
+        want = digit_s[1];
+        prefix |= pass == 0 ? bin << 21 : pass == 1 ? bin << 10 : bin;
+    }
+    const uint32_t T = prefix, r = want;
+
+    // ---- 2. per block: keys above T, keys equal to T, largest key; every block gets every block's ----
+    uint32_t my_gt = 0, my_eq = 0;
+    {
+        uint32_t mx = 0;
+#pragma unroll
+        for (int i = 0; i < kClE; ++i) {
+            my_gt += key[i] > T;
+            my_eq += key[i] == T;
+            mx = max(mx, key[i]);
+        }
+        uint32_t packed = my_gt | (my_eq << 16);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            packed += __shfl_xor_sync(0xFFFFFFFFu, packed, o);
+            mx = max(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+        }
+        if (lane == 0) {
+            atomicAdd(&red[0], packed & 0xFFFFu);
+            atomicAdd(&red[1], packed >> 16);
+            atomicMax(&red[2], mx);
+        }
+        __syncthreads();
+        if (tid < static_cast<int>(nblocks)) cluster.map_shared_rank(cta_cnt, tid)[rank] = make_uint4(red[0], red[1], red[2], 0u);
+    }
+    cluster.sync();
+
+    // ---- 3. ordered compaction ----
+    uint32_t gt_before = 0, eq_before = 0, kmax = 0;
+    for (uint32_t b = 0; b < nblocks; ++b) {
+        const uint4 c = cta_cnt[b];
+        gt_before += b < rank ? c.x : 0u;
+        eq_before += b < rank ? c.y : 0u;
+        kmax = max(kmax, c.z);
+    }
+    const uint32_t range = kmax - T;
+    const int passes = p.order == LSGD_ORDER_INDEX_ASC ? 0 : (32 - __clz(range) + kSortBits - 1) / kSortBits;
+    const bool direct = passes == 0;
+    const int R = p.sort_rounds;
+    const int tshift = 10 + (R == 1 ? 0 : R == 2 ? 1 : R == 4 ? 2 : 3);
+    const uint32_t tmask = (1u << tshift) - 1u;
+    const uint32_t St = p.sort_tiles;  // <= nblocks: sort tile b lives in block b
+    {
+        const uint32_t packed = block_exclusive_scan(my_gt | (my_eq << 16), warp_tot);
+        uint32_t gt_run = gt_before + (packed & 0xFFFFu);
+        uint32_t eq_run = eq_before + (packed >> 16);
+        const int64_t base = static_cast<int64_t>(rank) * kClTile + static_cast<int64_t>(tid) * kClE;
+#pragma unroll
+        for (int i = 0; i < kClE; ++i) {
+            const bool above = key[i] > T;
+            const bool tie = key[i] == T;
+            if (above || (tie && eq_run < r)) {
+                const uint32_t pos = gt_run + min(eq_run, r);
+                const int64_t j = base + i;
+                if (direct) {
+                    p.out_idx[pos] = static_cast<int32_t>(j);
+                    if (p.out_vals) p.out_vals[pos] = losses[j];
+                } else {
+                    cluster.map_shared_rank(pairs, pos >> tshift)[pos & tmask] = make_uint2(key[i], static_cast<uint32_t>(j));
+                }
+            }
+            gt_run += above;
+            eq_run += tie;
+        }
+    }
+    if (direct) return;  // nobody touches another block's shared memory after the barrier above
+    cluster.sync();
+
+    // ---- 4. stable LSD sort on u = kmax - key, 9 bits per pass; tile b = block b's pair buffer ----
+    uint32_t(*counters)[kCounterPitch] = reinterpret_cast<uint32_t(*)[kCounterPitch]>(dyn);
+    const uint32_t k = p.k;
+    const bool has_tile = rank < St;
+    const uint32_t first = (rank << tshift) + warp * (R * 32);  // global position of this warp's first entry
+    for (int pass = 0; pass < passes; ++pass) {
+        const bool last = pass == passes - 1;
+        const int shift = kSortBits * pass;
+        const uint2* pairs_in = pairs + (pass & 1) * kClTile;
+        uint2* pairs_out = pairs + ((pass + 1) & 1) * kClTile;
+        uint32_t skey[kSortMaxRounds], srank[kSortMaxRounds];
+        int32_t sidx[kSortMaxRounds];
+        if (has_tile) {
+            for (int i = tid; i < kWarps * kCounterPitch; i += kThreads) dyn[i] = 0;
+#pragma unroll
+            for (int rd = 0; rd < kSortMaxRounds; ++rd) {
+                const uint32_t e = first + rd * 32 + lane;
+                const bool live = rd < R && e < k;
+                const uint2 pr = live ? pairs_in[e & tmask] : make_uint2(0u, 0u);
+                skey[rd] = pr.x;
+                sidx[rd] = static_cast<int32_t>(pr.y);
+            }
+            __syncthreads();
+#pragma unroll
+            for (int rd = 0; rd < kSortMaxRounds; ++rd) {
+                if (rd < R) {
+                    const uint32_t e = first + rd * 32 + lane;
+                    const bool live = e < k;
+                    const uint32_t dd = ((kmax - skey[rd]) >> shift) & (kSortBins - 1);
+                    const uint32_t peers = match_digit(dd, live);
+                    const int leader = live ? __ffs(peers) - 1 : lane;
+                    uint32_t old = 0;
+                    if (live && lane == leader) {
+                        old = counters[warp][dd];
+                        counters[warp][dd] = old + __popc(peers);
+                    }
+                    old = __shfl_sync(0xFFFFFFFFu, old, leader);
+                    srank[rd] = old + __popc(peers & ((1u << lane) - 1u));
+                    __syncwarp();
+                }
+            }
+            __syncthreads();
+            {   // per digit, exclusive prefix of the warps' counts within each half of the block: thread (digit, half)
+                const int d = tid & (kSortBins - 1), h = tid / kSortBins;
+                constexpr int kHalf = kWarps / 2;
+                uint32_t c[kHalf];
+#pragma unroll
+                for (int u = 0; u < kHalf; ++u) c[u] = counters[kHalf * h + u][d];
+                uint32_t run = 0;
+#pragma unroll
+                for (int u = 0; u < kHalf; ++u) {
+                    counters[kHalf * h + u][d] = run;
+                    run += c[u];
+                }
+                half_cnt[h][d] = run;
+            }
+            __syncthreads();
+            // this tile's digit counts, into every block's copy of the count matrix
+            for (uint32_t i = tid; i < nblocks * kSortBins; i += kThreads) {
+                const uint32_t b = i / kSortBins, d = i % kSortBins;
+                cluster.map_shared_rank(mat, b)[rank * kSortBins + d] = half_cnt[0][d] + half_cnt[1][d];
+            }
+        }
+        cluster.sync();
+        if (has_tile) {
+            uint32_t before = 0;
+            if (tid < kSortBins) {
+                uint32_t total = 0;
+                for (uint32_t b = 0; b < St; ++b) {
+                    const uint32_t c = mat[b * kSortBins + tid];
+                    total += c;
+                    before += b < rank ? c : 0u;
+                }
+                tot_s[tid] = total;
+            }
+            __syncthreads();
+            if (warp == 0) {  // exclusive scan of the 512 digit totals, sixteen per lane
+                constexpr int kPer = kSortBins / 32;
+                uint32_t v[kPer], sum = 0;
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) {
+                    v[i] = tot_s[lane * kPer + i];
+                    sum += v[i];
+                }
+                uint32_t inc = sum;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                    if (lane >= o) inc += n;
+                }
+                uint32_t run = inc - sum;
+#pragma unroll
+                for (int i = 0; i < kPer; ++i) {
+                    tot_s[lane * kPer + i] = run;
+                    run += v[i];
+                }
+            }
+            __syncthreads();
+            if (tid < kSortBins) base_s[tid] = tot_s[tid] + before;
+            __syncthreads();
+#pragma unroll
+            for (int rd = 0; rd < kSortMaxRounds; ++rd) {
+                if (rd < R) {
+                    const uint32_t e = first + rd * 32 + lane;
+                    if (e < k) {
+                        const uint32_t dd = ((kmax - skey[rd]) >> shift) & (kSortBins - 1);
+                        const uint32_t pos = base_s[dd] + counters[warp][dd] + (warp >= kWarps / 2 ? half_cnt[0][dd] : 0u) + srank[rd];
+                        if (last) {
+                            p.out_idx[pos] = sidx[rd];
+                            if (p.out_vals) p.out_vals[pos] = losses[sidx[rd]];
+                        } else {
+                            cluster.map_shared_rank(pairs_out, pos >> tshift)[pos & tmask] = make_uint2(skey[rd], static_cast<uint32_t>(sidx[rd]));
+                        }
+                    }
+                }
+            }
+        }
+        if (!last) cluster.sync();  // after the last pass's exchange nobody touches another block's shared memory
     }
 }
 
@@ -640,9 +911,9 @@ small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int
     }
 }
 
-template <int E, bool CLUSTER>
+template <int E>
 cudaError_t launch_select(const SelectParams& p, int grid, cudaStream_t s) {
-    auto kernel = topk_select_kernel<E, CLUSTER>;
+    auto kernel = topk_select_kernel<E>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kDynSmemBytes));
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
@@ -650,24 +921,34 @@ cudaError_t launch_select(const SelectParams& p, int grid, cudaStream_t s) {
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kDynSmemBytes;
     cfg.stream = s;
-    cudaLaunchAttribute attr[2];
-    if (CLUSTER) {
-        // one cluster; it may be scheduled while the previous kernel of the stream drains (it waits for that
-        // kernel's completion before its first global access)
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = static_cast<unsigned>(grid);
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.numAttrs = 2;
-    } else {
-        attr[0].id = cudaLaunchAttributeCooperative;  // all blocks resident at once, or the launch is refused
-        attr[0].val.cooperative = 1;
-        cfg.numAttrs = 1;
-    }
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;  // all blocks resident at once, or the launch is refused
+    attr[0].val.cooperative = 1;
+    cfg.numAttrs = 1;
     cfg.attrs = attr;
     return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
+// One cluster of `grid` blocks; it may be scheduled while the previous kernel of the stream drains (it waits for
+// that kernel's completion before its first global access).
+cudaError_t launch_cluster(const SelectParams& p, int grid, cudaStream_t s) {
+    cudaError_t e = cudaFuncSetAttribute(topk_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kClSmemBytes));
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kClSmemBytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(grid);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 2;
+    cfg.attrs = attr;
+    return cudaLaunchKernelEx(&cfg, topk_cluster_kernel, p);
 }
 
 // Blocks of topk_select_kernel that can be resident at once on the current device (cached per device).
@@ -677,7 +958,7 @@ int resident_blocks() {
     if (cudaGetDevice(&dev) != cudaSuccess) return 1;
     int& c = cache[dev & 63];
     if (c == 0) {
-        auto kernel = topk_select_kernel<16, false>;
+        auto kernel = topk_select_kernel<16>;
         int per_sm = 0;
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kDynSmemBytes)) != cudaSuccess ||
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, kDynSmemBytes) != cudaSuccess || per_sm < 1)
@@ -704,14 +985,13 @@ cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order or
     p.ws = ws;
     p.hist0_ready = hist0_ready ? 1 : 0;
     const TestGeometry tg = test_geometry();
-    // One cluster of up to 8 blocks, 8,192 entries each, when the pool fits.
-    constexpr int64_t kClusterTile = int64_t{kThreads} * 8;
-    const int max_cluster = std::max(1, std::min(kMaxClusterBlocks, tg.max_ctas));
-    if (!tg.no_cluster && N <= kClusterTile * kMaxClusterBlocks) {
-        const int grid = static_cast<int>(std::min<int64_t>((N + kClusterTile - 1) / kClusterTile, max_cluster));
+    // One cluster of up to 8 blocks, 8,192 entries each, when the pool fits (and the test hook leaves it its blocks).
+    const int64_t cluster_blocks = (N + kClTile - 1) / kClTile;
+    if (!tg.no_cluster && cluster_blocks <= kMaxClusterBlocks && cluster_blocks <= tg.max_ctas) {
+        const int grid = static_cast<int>(cluster_blocks);
         p.sort_rounds = sort_rounds_for(k, grid);
         p.sort_tiles = static_cast<uint32_t>((k + 1024 * p.sort_rounds - 1) / (1024 * p.sort_rounds));
-        return launch_select<8, true>(p, grid, s);
+        return launch_cluster(p, grid, s);
     }
     const int resident = std::max(1, std::min(resident_blocks(), tg.max_ctas));
     p.sort_rounds = sort_rounds_for(k, std::min(resident, kSortDirectTiles));
@@ -719,9 +999,9 @@ cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order or
     auto tiles = [&](int e) { return (N + int64_t{kThreads} * e - 1) / (int64_t{kThreads} * e); };
     const int e = tiles(4) <= resident ? 4 : tiles(8) <= resident ? 8 : 16;
     const int grid = static_cast<int>(std::min<int64_t>(resident, std::max<int64_t>(tiles(e), p.sort_tiles)));
-    if (e == 4) return launch_select<4, false>(p, grid, s);
-    if (e == 8) return launch_select<8, false>(p, grid, s);
-    return launch_select<16, false>(p, grid, s);
+    if (e == 4) return launch_select<4>(p, grid, s);
+    if (e == 8) return launch_select<8>(p, grid, s);
+    return launch_select<16>(p, grid, s);
 }
 
 }  // namespace lsgd
