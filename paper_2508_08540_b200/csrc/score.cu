@@ -55,19 +55,20 @@ struct Elem<__nv_bfloat16> {
     __device__ static __nv_bfloat16 neg_inf_elem() { return __ushort_as_bfloat16(0xFF80u); }
 };
 
-// The selector's first radix digit, accumulated per CTA in shared memory.
+// The selector's first radix digit, accumulated per CTA in shared memory (or, with smem == nullptr, added
+// straight to the global histogram: kernels whose rows are long enough for one global atomic per row to be free).
 struct Hist0 {
     uint32_t* smem;
     uint32_t* global;
     __device__ void clear() {
-        if (global)
+        if (global && smem)
             for (int i = threadIdx.x; i < kSelBins; i += blockDim.x) smem[i] = 0;
     }
     __device__ void add(float loss) {
-        if (global) atomicAdd(&smem[loss_key(loss) >> 21], 1u);
+        if (global) atomicAdd(smem ? &smem[loss_key(loss) >> 21] : &global[loss_key(loss) >> 21], 1u);
     }
     __device__ void flush() {
-        if (global)
+        if (global && smem)
             for (int i = threadIdx.x; i < kSelBins; i += blockDim.x)
                 if (smem[i]) atomicAdd(&global[i], smem[i]);
     }
@@ -292,7 +293,7 @@ score_tiny_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
 // according to their length, and a lane reads chunks of that size, l, l + L, ...
 // of its row; otherwise it reads elements l, l + L, ...
 // ---------------------------------------------------------------------------
-constexpr int kGroupThreads = 256;
+constexpr int kGroupThreads = 128;
 constexpr int kGroupMaxRowBytes = 2048;
 constexpr int kGroupStages = 2;
 
@@ -401,7 +402,7 @@ __device__ __forceinline__ void chunk_sum_exp(const typename ChunkWord<CB>::type
 // the registers), one tile ahead of the one being reduced, so every CTA always has loads in flight; two stages
 // rather than three leave room for a third CTA per SM, which is worth more (measured).
 template <typename T, int L, int CB>
-__global__ void __launch_bounds__(kGroupThreads, 4)
+__global__ void __launch_bounds__(kGroupThreads, 8)
 score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
                         int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0,
                         int stage_bytes) {
@@ -409,9 +410,8 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
     constexpr bool VEC = CB > 0;          // rows start on CB-byte boundaries and are whole chunks (base 16-byte aligned)
     constexpr bool PADDED = CB == 16 && L < 8;
     extern __shared__ __align__(16) unsigned char group_smem[];
-    uint32_t* hist_s = reinterpret_cast<uint32_t*>(group_smem);
-    unsigned char* stages = group_smem + kSelBins * sizeof(uint32_t);
-    Hist0 h{hist_s, hist0};
+    unsigned char* stages = group_smem;
+    Hist0 h{nullptr, hist0};  // rows of more than 416 bytes: one global atomic per row costs nothing
     h.clear();
     const int row_bytes = C * static_cast<int>(sizeof(T));
     const int64_t tiles = (rows + R - 1) / R;
@@ -1028,7 +1028,7 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
             const int64_t nchunk = row_bytes / 16;
             const int64_t pitch = (cb == 16 && lanes < 8) ? 16 * (nchunk + ((lanes - nchunk) & 7)) : row_bytes;
             const int stage_bytes = static_cast<int>((tile_rows * pitch + 32 + 15) / 16 * 16);
-            const size_t smem = kSelBins * sizeof(uint32_t) + static_cast<size_t>(kGroupStages) * stage_bytes;
+            const size_t smem = static_cast<size_t>(kGroupStages) * stage_bytes;
             err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynSmem));
             if (err != cudaSuccess) return;
             const int64_t tiles = (rows + tile_rows - 1) / tile_rows;
@@ -1045,7 +1045,7 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
                 if constexpr (sizeof(T) == 2) go(score_group_rows_kernel<T, LN, 4>, LN);  // (4-byte chunks of fp32 are single elements)
             } else go(score_group_rows_kernel<T, LN, 0>, LN);
         };
-        // rows per tile (256 / L) times bytes per row: at most 32 KB per stage (64 x 512, 32 x 1024, 16 x 2048), plus padding
+        // rows per tile (128 / L) times bytes per row: at most 16 KB per stage (32 x 512, 16 x 1024, 8 x 2048), plus padding
         if (row_bytes <= 512) by_chunk(std::integral_constant<int, 4>{});
         else if (row_bytes <= 1024) by_chunk(std::integral_constant<int, 8>{});
         else by_chunk(std::integral_constant<int, 16>{});
