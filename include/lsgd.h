@@ -19,7 +19,11 @@
  *     synchronise, except lsgd_read_device_status.
  *   - Errors are reported by return value only.  Argument errors are found on
  *     the host before anything is launched, so a failing call has no effect on
- *     the device.  No kernel traps, and no kernel waits on another thread block.
+ *     the device.  No kernel traps.  One kernel has thread blocks that wait for
+ *     each other: the selector for pools above 65,536 entries, launched
+ *     cooperatively (all its blocks resident at once) with a barrier whose polls
+ *     are counted; if the count ever ran out the kernel would give up, leave its
+ *     outputs unspecified and record LSGD_ERR_TIMEOUT in the status block.
  *   - A size of zero (N == 0, k == 0, D == 0) is legal: the call returns LSGD_OK
  *     without launching anything.
  *   - Workspaces must be 256-byte aligned.  Their contents are scratch: they
@@ -50,7 +54,7 @@ typedef enum lsgd_status {
     LSGD_ERR_ALIGNMENT = 3,   /* pointer not aligned to its element size, workspace not to 256 B      */
     LSGD_ERR_WORKSPACE = 4,   /* ws_bytes smaller than the matching *_workspace_bytes query           */
     LSGD_ERR_CUDA = 5,        /* the CUDA runtime refused a launch or a memset                        */
-    LSGD_ERR_TIMEOUT = 6      /* reserved: a bounded device-side wait ran out (no kernel of this version waits) */
+    LSGD_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out (reported by lsgd_read_device_status)       */
 } lsgd_status;
 
 /* Element type of the logits. Labels are always int64, losses always fp32. */
@@ -126,6 +130,8 @@ LSGD_API lsgd_status lsgd_score_losses(const void* logits, lsgd_dtype dtype, con
  *   out_idx   device, [k] int32, the selected indices in `order`.
  *   out_vals  device, [k] fp32 or NULL: losses[out_idx[j]], bits unchanged.
  *   ws        device workspace of at least lsgd_topk_workspace_bytes(N, k).
+ * One kernel per call: pools of up to 1,024 entries in one thread block, up to
+ * 65,536 in one thread-block cluster, larger ones in a cooperative launch.
  */
 LSGD_API lsgd_status lsgd_topk_select(const float* losses, int64_t N, int64_t k, lsgd_order order,
                                       int32_t* out_idx, float* out_vals, void* ws, size_t ws_bytes,
@@ -331,8 +337,8 @@ LSGD_API lsgd_status lsgd_weights_from_steps(const int32_t* tau, int32_t P, floa
  * selection call left at the start of `ws`.  Synchronises `cuda_stream`.
  *   bad_label_count  host, out: tokens whose label was outside [0, C) and not
  *                    ignore_index in that call.
- * Returns LSGD_ERR_CUDA if the copy failed, else LSGD_OK (LSGD_ERR_TIMEOUT is reserved
- * for kernels with bounded device-side waits; this version has none).
+ * Returns LSGD_ERR_CUDA if the copy failed, LSGD_ERR_TIMEOUT if the selector's barrier
+ * gave up in that call (its outputs are then unspecified), else LSGD_OK.
  */
 LSGD_API lsgd_status lsgd_read_device_status(const void* ws, int32_t* bad_label_count, void* cuda_stream);
 

@@ -52,9 +52,13 @@ struct TopkWorkspace {       // device pointers carved out of the caller's works
 // Test hooks (environment, read at every launch): they change launch geometry only, never results.
 //   LSGD_TEST_MAX_CTAS=n     no kernel of the scorer or the selector uses more than n thread blocks
 //   LSGD_TEST_NO_CLUSTER=1   the selector never runs as a single cluster
+// and one that makes the cooperative selector's barrier give up, to test that path without harming the device:
+//   LSGD_TEST_PHANTOM_BLOCK=1  the barrier waits for one block more than exist, with a short poll limit (tens of
+//                              milliseconds): every block sets the timeout word and returns; outputs are unspecified
 struct TestGeometry {
     int max_ctas;      // INT_MAX when unset
     bool no_cluster;
+    bool phantom_block;
 };
 TestGeometry test_geometry();
 

@@ -195,3 +195,24 @@ def test_round_aggregation_stays_inside_its_guards(L, oracle, D, P, bf16):
     o64, _, _, mag = oracle.aggregate_round(reps, w, base)
     err = np.abs(out.cpu().numpy().astype(np.float64) - o64)
     assert (err <= 1e-6 * mag + 2.0 ** -24 * 1.01 * np.abs(o64)).all()
+
+
+def test_selector_barrier_gives_up_cleanly(L, oracle):
+    """The cooperative selector's barrier is bounded: made to wait for a thread block that does not exist (a test
+    hook; nothing on the device is harmed), every block gives up after its poll limit, the status block reports
+    LSGD_ERR_TIMEOUT, and the next call on the same context works."""
+    N, k = 200_003, 50_000
+    h = wl.loss_like_vector(77, N, dup_frac=0.01)
+    v = torch.from_numpy(h).cuda()
+    ws = L.workspace(L.topk_workspace_bytes(N, k))
+    os.environ["LSGD_TEST_PHANTOM_BLOCK"] = "1"
+    try:
+        L.topk_select(v, k, L.ORDER_LOSS_DESC, ws=ws)
+        with pytest.raises(L.LsgdError) as e:
+            L.read_device_status(ws)
+        assert e.value.status == L.ERR_TIMEOUT
+    finally:
+        del os.environ["LSGD_TEST_PHANTOM_BLOCK"]
+    idx, _ = L.topk_select(v, k, L.ORDER_LOSS_DESC, ws=ws)
+    assert L.read_device_status(ws) == 0
+    np.testing.assert_array_equal(idx.cpu().numpy(), oracle.topk(h, k, oracle.LOSS_DESC)[0])
