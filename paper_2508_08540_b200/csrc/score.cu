@@ -584,7 +584,8 @@ score_lane_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
     constexpr int ES = static_cast<int>(sizeof(T));
     constexpr int EPC = 16 / ES;  // elements per 16-byte chunk
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    unsigned char* ring = lane_smem + kSelBins * sizeof(uint32_t) + static_cast<size_t>(warp) * STAGES * stage_bytes;
+    // (the histogram's 8 KB are only there when a histogram is asked for)
+    unsigned char* ring = lane_smem + (hist0 ? kSelBins * sizeof(uint32_t) : 0) + static_cast<size_t>(warp) * STAGES * stage_bytes;
     const int row_bytes = C * ES;
     const int rc = PADDED ? row_bytes >> 4 : 1;  // chunks per row
     const int pitch = rc | 1;                     // odd: the eight lanes of a quarter-warp read eight different bank groups
@@ -975,7 +976,7 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
         auto go = [&](auto kernel, int threads, int stages) {
             const int64_t rc = row_bytes / 16;
             const int stage_bytes = static_cast<int>(cb == 16 ? 32 * (rc | 1) * 16 : (32 * row_bytes + 15) / 16 * 16);
-            const size_t smem = kSelBins * sizeof(uint32_t) + static_cast<size_t>(threads / 32) * stages * stage_bytes;
+            const size_t smem = (hist0 ? kSelBins * sizeof(uint32_t) : 0) + static_cast<size_t>(threads / 32) * stages * stage_bytes;
             err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynSmem));
             if (err != cudaSuccess) return;
             const int64_t want = ((rows + 31) / 32 + threads / 32 - 1) / (threads / 32);
@@ -1006,7 +1007,9 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
             else if (cb == 4) go(score_lane_rows_kernel<T, 0, 4, ST>, kLaneThreads, ST);
             else go(score_lane_rows_kernel<T, 0, 2, ST>, kLaneThreads, ST);
         };
-        if (32 * row_bytes <= 6144) by_unit(std::integral_constant<int, 3>{});
+        // warps per SM are what hides the latencies here, and the ring's size is what limits them: a third stage
+        // only where sixteen warps still fit (measured: 176-byte rows lose a quarter going from 12 to 8 warps per SM)
+        if (32 * row_bytes <= 4608) by_unit(std::integral_constant<int, 3>{});
         else by_unit(std::integral_constant<int, 2>{});
         return err;
     }
