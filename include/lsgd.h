@@ -96,9 +96,12 @@ LSGD_API size_t lsgd_score_topk_workspace_bytes(int64_t N, int64_t T, int64_t C,
  *
  *   logits  device, [N, T, C] row-major, contiguous, dtype `dtype`, aligned to
  *           its element size (16-byte alignment is faster, not required).
- *           Values must be finite with |x| <= 1e30 (the kernels form x * log2(e)
- *           in fp32 and start their running maxima at -1e30; beyond that range
- *           results are unspecified).  Rows whose label is ignore_index are not scored,
+ *           Values must be finite with |x| <= 1e8: the kernels work with
+ *           x * log2(e) rounded to fp32 and carry the rounding error of that
+ *           product for the row maximum along exactly, which needs it to stay
+ *           within the range of an exponent (it is at most 8 for |x| <= 1e8);
+ *           beyond that range results are unspecified.  Rows whose label is
+ *           ignore_index are not scored,
  *           and rows longer than 2 KB are then not read at all (shorter rows are
  *           loaded in contiguous tiles, ignored rows included; their values are
  *           not used).

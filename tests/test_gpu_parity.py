@@ -134,6 +134,27 @@ def test_score_closed_forms_and_small_losses(L, oracle):
         assert_losses_close(got, want, C)
 
 
+@pytest.mark.parametrize("C,dtype", [(10, "f32"), (32, "bf16"), (100, "f32"), (100, "bf16"), (500, "f32"), (1000, "bf16"), (5000, "f32"),
+                                     (9000, "bf16"), (70_001, "f32")])
+def test_score_at_the_documented_logit_bound(L, oracle, C, dtype):
+    """Logits as large as the header allows (|x| <= 1e8; here +-2^26, exact in bf16), in every scorer kernel: ties at
+    the top, the true class at the top, at the bottom and in between."""
+    big = np.float32(2.0 ** 26)
+    rng = np.random.default_rng(C)
+    N = 64
+    x = rng.choice(np.array([big, -big, big * np.float32(0.9921875), 0.0, 1.0, -3.0], np.float32), size=(N, C)).astype(np.float32)
+    x[:, 0] = big                    # every row has the bound itself ...
+    x[::2, C // 2] = big             # ... half of them twice
+    y = rng.integers(0, C, N)
+    y[:8] = 0                        # the true class is the maximum
+    y[8:16] = C // 2
+    xs = wl.f32_to_bf16_bits(x) if dtype == "bf16" else x
+    want, bad = oracle.score(xs, y)
+    assert bad == 0 and np.isfinite(want).all()
+    got = L.score_losses(dev_logits(xs), torch.from_numpy(y).cuda()).cpu().numpy()
+    assert_losses_close(got, want, C)
+
+
 @pytest.mark.parametrize("C,dtype", [(10, "f32"), (40, "bf16"), (100, "f32"), (102, "bf16"), (500, "f32"), (1000, "bf16"),
                                      (1500, "f32"), (5000, "bf16"), (30522, "bf16"), (70001, "f32")])
 @pytest.mark.parametrize("off", [0, 1, 3])
