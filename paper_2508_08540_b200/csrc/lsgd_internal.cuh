@@ -36,7 +36,6 @@ constexpr int kTile = 4096;               // smallest selection tile (the per-ti
 constexpr int kSmallN = 1024;             // pools up to this size are sorted by one CTA, one entry per thread
 constexpr int kSortBits = 9;              // digits of the stable LSD sort of the selected pairs
 constexpr int kSortBins = 1 << kSortBits;
-constexpr int kSortPasses = 4;            // at most: 4 x 9 bits cover a 32-bit key range
 constexpr int kSortMaxRounds = 8;         // a sort tile holds 1024 R entries, R in {1, 2, 4, 8}
 constexpr int kSortDirectTiles = 256;     // the launcher grows R before it uses more sort tiles than this
 constexpr int kMaxClusterBlocks = 8;      // portable cluster size: pools of up to 8 x 8,192 entries run as one cluster

@@ -23,7 +23,9 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <mutex>
 #include <type_traits>
+#include <vector>
 
 #include "lsgd_internal.cuh"
 
@@ -474,9 +476,9 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
         __syncwarp();
         float m = -1e30f, s = 0.f;
         if constexpr (VEC && L >= 8) {
-            // A lane's share of a row is at most 128 bytes (rows of up to 512, 1024, 2048 bytes over 4, 8, 16
-            // lanes): it is read from shared memory once, into registers, and both passes run from there, fully
-            // unrolled.  Round i (chunks i L .. i L + L - 1) is skipped by the whole warp once it is past the row.
+            // A lane's share of a row is at most 128 bytes (rows of up to 1024 and 2048 bytes over 8 and 16 lanes:
+            // the launcher never gives this path longer ones): it is read from shared memory once, into registers,
+            // and both passes run from there, fully unrolled.  Round i (chunks i L .. i L + L - 1) is skipped by the whole warp once it is past the row.
             constexpr int CBV = VEC ? CB : 16;
             constexpr int kMaxCh = 128 / CBV;
             using Word = typename ChunkWord<CBV>::type;
@@ -953,14 +955,35 @@ seq_mean_kernel(const float* __restrict__ token_loss, const int64_t* __restrict_
     h.flush();
 }
 
+// Resident blocks per multiprocessor of `kernel` at this block size and dynamic shared memory.  The answer (and
+// the one-time opt-in to large dynamic shared memory) is remembered per device, kernel and size: the runtime calls
+// behind it cost microseconds of host time, which a small pool's whole call is measured in.
 template <typename K>
-int blocks_per_sm(K kernel, int threads, size_t smem) {
+int blocks_per_sm(K kernel, int threads, size_t smem, bool large_smem = false) {
+    struct Entry {
+        const void* fn;
+        int dev, threads, blocks;
+        size_t smem;
+    };
+    static std::mutex mu;
+    static std::vector<Entry> known;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const void* fn = reinterpret_cast<const void*>(kernel);
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        for (const Entry& e : known)
+            if (e.fn == fn && e.dev == dev && e.threads == threads && e.smem == smem) return e.blocks;
+    }
+    if (large_smem && cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(227 * 1024)) != cudaSuccess)
+        return 0;
     int b = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kernel, threads, smem) != cudaSuccess || b < 1) b = 1;
+    std::lock_guard<std::mutex> lock(mu);
+    known.push_back(Entry{fn, dev, threads, b, smem});
     return b;
 }
 
-constexpr size_t kMaxDynSmem = 227 * 1024;
 
 template <typename T>
 cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, int64_t C, int64_t ignore_index,
@@ -977,10 +1000,13 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
             const int64_t rc = row_bytes / 16;
             const int stage_bytes = static_cast<int>(cb == 16 ? 32 * (rc | 1) * 16 : (32 * row_bytes + 15) / 16 * 16);
             const size_t smem = (hist0 ? kSelBins * sizeof(uint32_t) : 0) + static_cast<size_t>(threads / 32) * stages * stage_bytes;
-            err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynSmem));
-            if (err != cudaSuccess) return;
+            const int bps = blocks_per_sm(kernel, threads, smem, true);
+            if (bps < 1) {
+                err = cudaErrorInvalidValue;
+                return;
+            }
             const int64_t want = ((rows + 31) / 32 + threads / 32 - 1) / (threads / 32);
-            const int grid = static_cast<int>(std::min({want, static_cast<int64_t>(sms) * blocks_per_sm(kernel, threads, smem), max_ctas}));
+            const int grid = static_cast<int>(std::min({want, static_cast<int64_t>(sms) * bps, max_ctas}));
             kernel<<<grid, threads, smem, s>>>(logits, labels, rows, static_cast<int>(C), ignore_index, row_loss, status,
                                                hist0, stage_bytes);
             err = cudaGetLastError();
@@ -1032,10 +1058,13 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
             const int64_t pitch = (cb == 16 && lanes < 8) ? 16 * (nchunk + ((lanes - nchunk) & 7)) : row_bytes;
             const int stage_bytes = static_cast<int>((tile_rows * pitch + 32 + 15) / 16 * 16);
             const size_t smem = static_cast<size_t>(kGroupStages) * stage_bytes;
-            err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynSmem));
-            if (err != cudaSuccess) return;
+            const int bps = blocks_per_sm(kernel, kGroupThreads, smem, true);
+            if (bps < 1) {
+                err = cudaErrorInvalidValue;
+                return;
+            }
             const int64_t tiles = (rows + tile_rows - 1) / tile_rows;
-            const int grid = static_cast<int>(std::min({tiles, static_cast<int64_t>(sms) * blocks_per_sm(kernel, kGroupThreads, smem), max_ctas}));
+            const int grid = static_cast<int>(std::min({tiles, static_cast<int64_t>(sms) * bps, max_ctas}));
             kernel<<<grid, kGroupThreads, smem, s>>>(logits, labels, rows, static_cast<int>(C), ignore_index, row_loss,
                                                      status, hist0, stage_bytes);
             err = cudaGetLastError();
@@ -1048,8 +1077,10 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
                 if constexpr (sizeof(T) == 2) go(score_group_rows_kernel<T, LN, 4>, LN);  // (4-byte chunks of fp32 are single elements)
             } else go(score_group_rows_kernel<T, LN, 0>, LN);
         };
-        // rows per tile (128 / L) times bytes per row: at most 16 KB per stage (32 x 512, 16 x 1024, 8 x 2048), plus padding
-        if (row_bytes <= 512) by_chunk(std::integral_constant<int, 4>{});
+        // rows per tile (128 / L) times bytes per row: at most 25 KB per stage (32 x 800, 16 x 1024, 8 x 2048), plus padding.
+        // As few lanes per row as the row length allows: the per-row work is shared by 32 / L rows of a warp (measured
+        // at 600 and 800 bytes: 4 lanes 0.74-0.98 of the copy rate against 0.61-0.96 with 8; at 1000 bytes 8 lanes win)
+        if (row_bytes <= 800) by_chunk(std::integral_constant<int, 4>{});
         else if (row_bytes <= 1024) by_chunk(std::integral_constant<int, 8>{});
         else by_chunk(std::integral_constant<int, 16>{});
         return err;

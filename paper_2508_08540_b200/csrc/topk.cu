@@ -32,6 +32,8 @@
 #include <cooperative_groups.h>
 
 #include <algorithm>
+#include <mutex>
+#include <vector>
 
 #include "lsgd_internal.cuh"
 
@@ -95,7 +97,7 @@ namespace {
 
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
-constexpr int kCounterPitch = kSortBins + 1;  // odd pitch: a warp can read one bin of all 32 rows without bank conflicts
+constexpr int kCounterPitch = kSortBins;      // one row of digit counters per warp
 constexpr size_t kDynSmemBytes = sizeof(uint32_t) * kWarps * kCounterPitch;
 constexpr uint32_t kMaxPolls = 1u << 21;      // barrier polls before a block gives up (seconds; never reached when all blocks are resident)
 
@@ -913,10 +915,36 @@ small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int
     }
 }
 
+// Opts `kernel` in to `bytes` of dynamic shared memory, once per kernel and device (the call costs host time at
+// every launch otherwise).  The kernels share one function type, so the memo is keyed by the function's address.
+template <typename K>
+cudaError_t allow_dynamic_smem(K kernel, size_t bytes) {
+    struct Entry {
+        const void* fn;
+        int dev;
+    };
+    static std::mutex mu;
+    static std::vector<Entry> done;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const void* fn = reinterpret_cast<const void*>(kernel);
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        for (const Entry& d : done)
+            if (d.fn == fn && d.dev == dev) return cudaSuccess;
+    }
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    done.push_back(Entry{fn, dev});
+    return cudaSuccess;
+}
+
 template <int E>
 cudaError_t launch_select(const SelectParams& p, int grid, cudaStream_t s) {
     auto kernel = topk_select_kernel<E>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kDynSmemBytes));
+    cudaError_t e = allow_dynamic_smem(kernel, kDynSmemBytes);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
@@ -934,7 +962,7 @@ cudaError_t launch_select(const SelectParams& p, int grid, cudaStream_t s) {
 // One cluster of `grid` blocks; it may be scheduled while the previous kernel of the stream drains (it waits for
 // that kernel's completion before its first global access).
 cudaError_t launch_cluster(const SelectParams& p, int grid, cudaStream_t s) {
-    cudaError_t e = cudaFuncSetAttribute(topk_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kClSmemBytes));
+    cudaError_t e = allow_dynamic_smem(topk_cluster_kernel, kClSmemBytes);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
