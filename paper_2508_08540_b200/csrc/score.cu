@@ -14,12 +14,14 @@
 // cancels against the same rounded product in the last step (see loss_without_true_class).
 //
 // Row shapes and their kernels (all bound by the bytes of the logits):
-//   tiny rows   (C <= 32)         one thread per row out of a shared-memory tile
-//   small rows  (<= 2 KB)         4, 8 or 16 lanes per row out of a shared-memory tile
-//   medium rows (<= 256 KB)       one warp per row, streamed through registers with a running (max, sum)
-//   anything longer               one CTA per row, two passes over global memory
+//   short rows  (<= 416 B, or <= 32 elements)   one LANE per row: a warp copies 32 rows into its own shared-memory ring
+//   small rows  (<= 2 KB)                        4, 8 or 16 lanes per row out of a block's shared-memory tile
+//   medium rows (<= 256 KB)                      one warp per row, streamed through registers with a running (max, sum)
+//   anything longer                              one CTA per row, two passes over global memory
+// (a pool whose base is not 16-byte aligned takes the lane-group kernel or, for rows of at most 32 elements, a
+// thread-per-row kernel with element-wise staging).
 // Rows whose label is ignore_index are never scored; the kernels for medium and longer rows do not even
-// read them (tiny and small rows are copied tile-wise, ignored rows included).
+// read them (short and small rows are copied block-wise, ignored rows included).
 #include <cuda_bf16.h>
 
 #include <algorithm>
@@ -286,7 +288,7 @@ score_tiny_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
 }
 
 // ---------------------------------------------------------------------------
-// Small rows (C > 32, at most 2 KB): a CTA copies a tile of consecutive rows (one
+// Small rows (417 bytes to 2 KB; shorter ones of an unaligned pool): a CTA copies a tile of consecutive rows (one
 // contiguous, 16-byte-aligned-superset byte range) into shared memory with
 // vector loads; groups of L lanes then own one row each and read it from there.
 // One warp per row would spend most of its instructions on 32-lane reductions
