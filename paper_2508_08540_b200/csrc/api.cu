@@ -22,12 +22,13 @@ int sm_count() {
 }
 
 TestGeometry test_geometry() {
-    TestGeometry g{2147483647, false, false};
+    TestGeometry g{2147483647, false, false, false};
     if (const char* v = std::getenv("LSGD_TEST_MAX_CTAS")) {
         const long n = std::strtol(v, nullptr, 10);
         if (n > 0 && n < 2147483647) g.max_ctas = static_cast<int>(n);
     }
     if (const char* v = std::getenv("LSGD_TEST_NO_CLUSTER")) g.no_cluster = v[0] == '1';
+    if (const char* v = std::getenv("LSGD_TEST_NARROW_CLUSTER")) g.narrow_cluster = v[0] == '1';
     if (const char* v = std::getenv("LSGD_TEST_PHANTOM_BLOCK")) g.phantom_block = v[0] == '1';
     return g;
 }

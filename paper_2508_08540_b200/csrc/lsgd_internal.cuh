@@ -38,7 +38,7 @@ constexpr int kSortBits = 9;              // digits of the stable LSD sort of th
 constexpr int kSortBins = 1 << kSortBits;
 constexpr int kSortMaxRounds = 8;         // a sort tile holds 1024 R entries, R in {1, 2, 4, 8}
 constexpr int kSortDirectTiles = 256;     // the launcher grows R before it uses more sort tiles than this
-constexpr int kMaxClusterBlocks = 8;      // portable cluster size: pools of up to 8 x 8,192 entries run as one cluster
+constexpr int kMaxClusterBlocks = 8;      // pools of up to 8 x 8,192 entries run as one cluster (of 16 x 4,096 where the device allows)
 
 struct TopkWorkspace {       // device pointers carved out of the caller's workspace
     StatusBlock* status;
@@ -51,12 +51,14 @@ struct TopkWorkspace {       // device pointers carved out of the caller's works
 // Test hooks (environment, read at every launch): they change launch geometry only, never results.
 //   LSGD_TEST_MAX_CTAS=n     no kernel of the scorer or the selector uses more than n thread blocks
 //   LSGD_TEST_NO_CLUSTER=1   the selector never runs as a single cluster
+//   LSGD_TEST_NARROW_CLUSTER=1  ... and when it does, as 8,192-entry blocks (the variant for devices without 16-block clusters)
 // and one that makes the cooperative selector's barrier give up, to test that path without harming the device:
 //   LSGD_TEST_PHANTOM_BLOCK=1  the barrier waits for one block more than exist, with a short poll limit (tens of
 //                              milliseconds): every block sets the timeout word and returns; outputs are unspecified
 struct TestGeometry {
     int max_ctas;      // INT_MAX when unset
     bool no_cluster;
+    bool narrow_cluster;
     bool phantom_block;
 };
 TestGeometry test_geometry();

@@ -229,6 +229,13 @@ __device__ __forceinline__ void load_keys(const float* __restrict__ losses, int6
     }
 }
 
+// The loss a key came from, where the key says it all; -0/+0 and NaNs (their sign and payload are not in the key) are
+// read back from the table.
+__device__ __forceinline__ float loss_of_key(uint32_t key, const float* __restrict__ losses, int32_t i) {
+    if (key == 0x80000000u || key == 0xFFFFFFFFu) return losses[i];
+    return __uint_as_float((key & 0x80000000u) ? key & 0x7FFFFFFFu : ~key);
+}
+
 // Lanes of the warp whose 9-bit digit equals this lane's, among the lanes with `live` set (0 for a lane that is
 // not live).  Ten votes; cheaper here than the generic match instruction.
 __device__ __forceinline__ uint32_t match_digit(uint32_t d, bool live) {
@@ -552,7 +559,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
                         const uint32_t pos = base_s[dd] + counters[warp][dd] + (warp >= kWarps / 2 ? half_cnt[0][dd] : 0u) + rank[rd];
                         if (last) {
                             p.out_idx[pos] = idx[rd];
-                            if (p.out_vals) p.out_vals[pos] = losses[idx[rd]];
+                            if (p.out_vals) p.out_vals[pos] = loss_of_key(key[rd], losses, idx[rd]);
                         } else {
                             __stcg(pairs_out + pos, make_uint2(key[rd], static_cast<uint32_t>(idx[rd])));
                         }
@@ -565,30 +572,38 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
 }
 
 // ---------------------------------------------------------------------------
-// Pools of up to kMaxClusterBlocks x 8,192 entries: the same algorithm as ONE thread-block cluster, everything
-// that blocks exchange kept in (distributed) shared memory.  Block b owns entries [8192 b, 8192 b + 8192) of the
-// pool (in registers) and sort tile b.  Digit histograms are added into block 0's shared memory and read from
+// Pools of up to 65,536 entries: the same algorithm as ONE thread-block cluster, everything that blocks exchange
+// kept in (distributed) shared memory.  Block b owns a slice of 4,096 or 8,192 consecutive entries of the pool (in
+// registers) and sort tile b.  Digit histograms are added into block 0's shared memory and read from
 // there by every block; per-block counts, the sort's digit counts and the (key, index) pairs themselves are
 // written straight into the destination block's shared memory.  The barrier is the cluster's hardware barrier.
 // ---------------------------------------------------------------------------
 namespace cg = cooperative_groups;
 
-constexpr int kClE = 8;
-constexpr int kClTile = kThreads * kClE;
-constexpr size_t kClCountersBytes = sizeof(uint32_t) * kWarps * kCounterPitch;
-constexpr size_t kClPairsBytes = sizeof(uint2) * 2 * kClTile;
-constexpr size_t kClMatBytes = sizeof(uint32_t) * kMaxClusterBlocks * kSortBins;
-constexpr size_t kClSmemBytes = kClCountersBytes + kClPairsBytes + kClMatBytes + sizeof(uint4) * kMaxClusterBlocks;
-static_assert(kClCountersBytes % 16 == 0, "the pair buffers start 16-byte aligned");
-static_assert(sizeof(uint32_t) * kSelPasses * kSelBins <= kClPairsBytes / 2, "the selection's histograms fit in the first pair buffer");
+// CE keys per thread (blocks of 1024 CE entries), at most CB blocks: 4 x 16 (a cluster of more than 8 blocks needs the
+// device's consent, see launch_topk) or 8 x 8.
+template <int CE, int CB>
+struct ClusterLayout {
+    static constexpr int kTile = kThreads * CE;
+    static constexpr size_t kCountersBytes = sizeof(uint32_t) * kWarps * kCounterPitch;
+    static constexpr size_t kPairsBytes = sizeof(uint2) * 2 * kTile;
+    static constexpr size_t kMatBytes = sizeof(uint32_t) * CB * kSortBins;
+    static constexpr size_t kSmemBytes = kCountersBytes + kPairsBytes + kMatBytes + sizeof(uint4) * CB;
+    static_assert(kCountersBytes % 16 == 0, "the pair buffers start 16-byte aligned");
+    static_assert(sizeof(uint32_t) * kSelPasses * kSelBins <= kPairsBytes / 2, "the selection's histograms fit in the first pair buffer");
+    static_assert(kTile <= 1024 * kSortMaxRounds, "a block's pairs are one sort tile");
+};
 
+template <int CE, int CB>
 __global__ void __launch_bounds__(kThreads, 1) topk_cluster_kernel(const __grid_constant__ SelectParams p) {
+    using Lay = ClusterLayout<CE, CB>;
+    constexpr int kClE = CE, kClTile = Lay::kTile;
     extern __shared__ __align__(16) unsigned char cl_smem[];
-    uint32_t* dyn = reinterpret_cast<uint32_t*>(cl_smem);                                   // hist_s, later counters
-    uint2* pairs = reinterpret_cast<uint2*>(cl_smem + kClCountersBytes);                     // [2][kClTile]
-    uint32_t* acc_hist = reinterpret_cast<uint32_t*>(pairs);                                 // block 0, selection only: [3][kSelBins]
-    uint32_t* mat = reinterpret_cast<uint32_t*>(cl_smem + kClCountersBytes + kClPairsBytes);  // [blocks][kSortBins]
-    uint4* cta_cnt = reinterpret_cast<uint4*>(cl_smem + kClCountersBytes + kClPairsBytes + kClMatBytes);
+    uint32_t* dyn = reinterpret_cast<uint32_t*>(cl_smem);                                          // hist_s, later counters
+    uint2* pairs = reinterpret_cast<uint2*>(cl_smem + Lay::kCountersBytes);                         // [2][kClTile]
+    uint32_t* acc_hist = reinterpret_cast<uint32_t*>(pairs);                                        // block 0, selection only: [3][kSelBins]
+    uint32_t* mat = reinterpret_cast<uint32_t*>(cl_smem + Lay::kCountersBytes + Lay::kPairsBytes);   // [blocks][kSortBins]
+    uint4* cta_cnt = reinterpret_cast<uint4*>(cl_smem + Lay::kCountersBytes + Lay::kPairsBytes + Lay::kMatBytes);
     __shared__ uint32_t warp_tot[kWarps + 1];
     __shared__ uint32_t result[2];
     __shared__ uint32_t red[3];
@@ -603,7 +618,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_cluster_kernel(const __grid_
 
     for (int i = tid; i < kSelBins; i += kThreads) hist_s[i] = 0;
     for (int i = tid; i < kSelPasses * kSelBins; i += kThreads) acc_hist[i] = 0;
-    for (int i = tid; i < kMaxClusterBlocks * kSortBins; i += kThreads) mat[i] = 0;
+    for (int i = tid; i < CB * kSortBins; i += kThreads) mat[i] = 0;
     if (tid < 3) red[tid] = 0;
     cluster.sync();          // every block's accumulators are clear before anybody adds to them
     grid_dependency_wait();  // the losses (and the scorer's histogram) are complete from here on
@@ -830,7 +845,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_cluster_kernel(const __grid_
                         const uint32_t pos = base_s[dd] + counters[warp][dd] + (warp >= kWarps / 2 ? half_cnt[0][dd] : 0u) + srank[rd];
                         if (last) {
                             p.out_idx[pos] = sidx[rd];
-                            if (p.out_vals) p.out_vals[pos] = losses[sidx[rd]];
+                            if (p.out_vals) p.out_vals[pos] = loss_of_key(skey[rd], losses, sidx[rd]);
                         } else {
                             cluster.map_shared_rank(pairs_out, pos >> tshift)[pos & tmask] = make_uint2(skey[rd], static_cast<uint32_t>(sidx[rd]));
                         }
@@ -961,15 +976,13 @@ cudaError_t launch_select(const SelectParams& p, int grid, cudaStream_t s) {
 
 // One cluster of `grid` blocks; it may be scheduled while the previous kernel of the stream drains (it waits for
 // that kernel's completion before its first global access).
-cudaError_t launch_cluster(const SelectParams& p, int grid, cudaStream_t s) {
-    cudaError_t e = allow_dynamic_smem(topk_cluster_kernel, kClSmemBytes);
-    if (e != cudaSuccess) return e;
+template <int CE, int CB>
+cudaLaunchConfig_t cluster_config(int grid, cudaStream_t s, cudaLaunchAttribute (&attr)[2]) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = kClSmemBytes;
+    cfg.dynamicSmemBytes = ClusterLayout<CE, CB>::kSmemBytes;
     cfg.stream = s;
-    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = static_cast<unsigned>(grid);
     attr[0].val.clusterDim.y = 1;
@@ -978,7 +991,40 @@ cudaError_t launch_cluster(const SelectParams& p, int grid, cudaStream_t s) {
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.numAttrs = 2;
     cfg.attrs = attr;
-    return cudaLaunchKernelEx(&cfg, topk_cluster_kernel, p);
+    return cfg;
+}
+
+template <int CE, int CB>
+cudaError_t launch_cluster(const SelectParams& p, int grid, cudaStream_t s) {
+    cudaError_t e = allow_dynamic_smem(topk_cluster_kernel<CE, CB>, ClusterLayout<CE, CB>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    cudaLaunchAttribute attr[2];
+    cudaLaunchConfig_t cfg = cluster_config<CE, CB>(grid, s, attr);
+    return cudaLaunchKernelEx(&cfg, topk_cluster_kernel<CE, CB>, p);
+}
+
+// Whether this device runs the 16-block cluster variant (clusters of more than 8 blocks are an opt-in, and the device
+// must be able to co-schedule 16 blocks of this size in one cluster).  Asked once per device.
+bool wide_cluster_ok() {
+    static std::mutex mu;
+    static int known[64] = {0};  // 0 unknown, 1 yes, 2 no
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    int& k = known[dev & 63];
+    if (k == 0) {
+        k = 2;
+        auto kernel = topk_cluster_kernel<4, 16>;
+        if (allow_dynamic_smem(kernel, ClusterLayout<4, 16>::kSmemBytes) == cudaSuccess &&
+            cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+            cudaLaunchAttribute attr[2];
+            cudaLaunchConfig_t cfg = cluster_config<4, 16>(16, nullptr, attr);
+            int clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg) == cudaSuccess && clusters >= 1) k = 1;
+        }
+        cudaGetLastError();  // a refusal above is an answer, not an error of the call being made
+    }
+    return k == 1;
 }
 
 // Blocks of topk_select_kernel that can be resident at once on the current device (cached per device).
@@ -1017,13 +1063,17 @@ cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order or
     p.barrier_parties = 0;
     p.barrier_polls = kMaxPolls;
     const TestGeometry tg = test_geometry();
-    // One cluster of up to 8 blocks, 8,192 entries each, when the pool fits (and the test hook leaves it its blocks).
-    const int64_t cluster_blocks = (N + kClTile - 1) / kClTile;
-    if (!tg.no_cluster && cluster_blocks <= kMaxClusterBlocks && cluster_blocks <= tg.max_ctas) {
-        const int grid = static_cast<int>(cluster_blocks);
-        p.sort_rounds = sort_rounds_for(k, grid);
-        p.sort_tiles = static_cast<uint32_t>((k + 1024 * p.sort_rounds - 1) / (1024 * p.sort_rounds));
-        return launch_cluster(p, grid, s);
+    // One cluster when the pool fits (and the test hook leaves it its blocks): up to 16 blocks of 4,096 entries
+    // where the device takes clusters that wide, else up to 8 blocks of 8,192.
+    if (!tg.no_cluster && N <= int64_t{kMaxClusterBlocks} * 8192) {
+        const int64_t blocks4 = (N + 4095) / 4096, blocks8 = (N + 8191) / 8192;
+        const bool wide = blocks4 <= tg.max_ctas && !tg.narrow_cluster && (blocks4 <= 8 || wide_cluster_ok());
+        const int grid = static_cast<int>(wide ? blocks4 : blocks8);
+        if (grid <= tg.max_ctas) {
+            p.sort_rounds = sort_rounds_for(k, grid);
+            p.sort_tiles = static_cast<uint32_t>((k + 1024 * p.sort_rounds - 1) / (1024 * p.sort_rounds));
+            return wide ? launch_cluster<4, 16>(p, grid, s) : launch_cluster<8, 8>(p, grid, s);
+        }
     }
     const int resident = std::max(1, std::min(resident_blocks(), tg.max_ctas));
     p.sort_rounds = sort_rounds_for(k, std::min(resident, kSortDirectTiles));

@@ -31,14 +31,16 @@ def L():
 
 
 @contextmanager
-def geometry(max_ctas=None, no_cluster=False):
+def geometry(max_ctas=None, no_cluster=False, narrow_cluster=False):
     """The library reads these at every launch; they change grid sizes only."""
-    old = {k: os.environ.get(k) for k in ("LSGD_TEST_MAX_CTAS", "LSGD_TEST_NO_CLUSTER")}
+    old = {k: os.environ.get(k) for k in ("LSGD_TEST_MAX_CTAS", "LSGD_TEST_NO_CLUSTER", "LSGD_TEST_NARROW_CLUSTER")}
     try:
         if max_ctas is not None:
             os.environ["LSGD_TEST_MAX_CTAS"] = str(max_ctas)
         if no_cluster:
             os.environ["LSGD_TEST_NO_CLUSTER"] = "1"
+        if narrow_cluster:
+            os.environ["LSGD_TEST_NARROW_CLUSTER"] = "1"
         yield
     finally:
         for k, v in old.items():
@@ -95,8 +97,8 @@ def test_selector_is_the_same_in_every_geometry(L, oracle, N, k, order):
     h = wl.loss_like_vector(N ^ k, N, dup_frac=0.02, specials=True)
     v = torch.from_numpy(h).cuda()
     want_idx, want_vals = oracle.topk(h, k, order)
-    runs = [dict(), dict(no_cluster=True), dict(max_ctas=3), dict(max_ctas=1), dict(no_cluster=True, max_ctas=5),
-            dict(no_cluster=True, max_ctas=1)]
+    runs = [dict(), dict(narrow_cluster=True), dict(no_cluster=True), dict(max_ctas=3), dict(max_ctas=1), dict(max_ctas=8),
+            dict(no_cluster=True, max_ctas=5), dict(no_cluster=True, max_ctas=1)]
     for kw in runs:
         with geometry(**kw):
             idx, vals = L.topk_select(v, k, order)
@@ -120,7 +122,7 @@ def test_selector_sort_pass_counts(L, oracle):
             h[100:110] = np.nan
         h = np.where(np.isfinite(h) | np.isnan(h), h, np.float32(3.0)).astype(np.float32)
         v = torch.from_numpy(h).cuda()
-        for kw in (dict(), dict(no_cluster=True)):
+        for kw in (dict(), dict(narrow_cluster=True), dict(no_cluster=True)):
             with geometry(**kw):
                 idx, vals = L.topk_select(v, k, L.ORDER_LOSS_DESC)
             want_idx, want_vals = oracle.topk(h, k, oracle.LOSS_DESC)
@@ -134,7 +136,7 @@ def test_fused_call_is_the_same_in_every_geometry(L, oracle, N, T, C, dtype, k):
     xd, yd = dev_logits(x), torch.from_numpy(y).cuda()
     ref_l, ref_i, ref_v = L.score_topk(xd, yd, k, L.ORDER_LOSS_DESC)
     np.testing.assert_array_equal(ref_i.cpu().numpy(), oracle.topk(ref_l.cpu().numpy(), k, oracle.LOSS_DESC)[0])
-    for kw in (dict(max_ctas=2), dict(no_cluster=True), dict(no_cluster=True, max_ctas=3)):
+    for kw in (dict(max_ctas=2), dict(narrow_cluster=True), dict(no_cluster=True), dict(no_cluster=True, max_ctas=3)):
         with geometry(**kw):
             l, i, v = L.score_topk(xd, yd, k, L.ORDER_LOSS_DESC)
         assert torch.equal(l.view(torch.int32), ref_l.view(torch.int32)) and torch.equal(i, ref_i)
