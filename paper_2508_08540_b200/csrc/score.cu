@@ -624,15 +624,18 @@ score_lane_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
         return y;
     };
 
-    int64_t yq[STAGES - 1];
+    int64_t yq[STAGES > 1 ? STAGES - 1 : 1];  // labels of the blocks in flight
 #pragma unroll
     for (int i = 0; i < STAGES - 1; ++i) yq[i] = issue(i);
     for (int64_t i = 0; i < mine; ++i) {
         const int64_t y_new = issue(i + STAGES - 1);
-        const int64_t y = yq[0];
+        int64_t y = y_new;  // STAGES == 1: no block ahead (pools so small that every warp gets at most one block)
+        if constexpr (STAGES > 1) {
+            y = yq[0];
 #pragma unroll
-        for (int q = 0; q + 1 < STAGES - 1; ++q) yq[q] = yq[q + 1];
-        yq[STAGES - 2] = y_new;
+            for (int q = 0; q + 1 < STAGES - 1; ++q) yq[q] = yq[q + 1];
+            yq[STAGES - 2] = y_new;
+        }
         cp_async_wait<STAGES - 1>();
         __syncwarp();  // every lane's copies of block i have landed
         const int64_t row0 = (gw + i * nw) << 5;
@@ -1035,6 +1038,17 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
             else if (cb == 4) go(score_lane_rows_kernel<T, 0, 4, ST>, kLaneThreads, ST);
             else go(score_lane_rows_kernel<T, 0, 2, ST>, kLaneThreads, ST);
         };
+        // A pool so small that, with a single stage per warp, every block of 32 rows gets a warp of its own at once:
+        // nothing to pipeline, and twice the warps are resident (a CIFAR-sized pool is scored in one wave).
+        {
+            const int64_t stage1 = cb == 16 ? 32 * ((row_bytes / 16) | 1) * 16 : (32 * row_bytes + 15) / 16 * 16;
+            const int64_t per_cta = (hist0 ? kSelBins * sizeof(uint32_t) : 0) + (kLaneThreads / 32) * stage1 + 1024;
+            const int64_t ctas = std::min<int64_t>(32, (227 * 1024) / per_cta);
+            if ((rows + 31) / 32 <= static_cast<int64_t>(sms) * ctas * (kLaneThreads / 32) && max_ctas >= static_cast<int64_t>(sms) * ctas) {
+                by_unit(std::integral_constant<int, 1>{});
+                return err;
+            }
+        }
         // warps per SM are what hides the latencies here, and the ring's size is what limits them: a third stage
         // only where sixteen warps still fit (measured: 176-byte rows lose a quarter going from 12 to 8 warps per SM)
         if (32 * row_bytes <= 4608) by_unit(std::integral_constant<int, 3>{});

@@ -229,6 +229,28 @@ __device__ __forceinline__ void load_keys(const float* __restrict__ losses, int6
     }
 }
 
+// Where each digit's run starts for a tile: base_s[d] = (entries of smaller digits, all tiles) + before_d.  Called by
+// every thread of the block; thread d < kSortBins passes digit d's total over all tiles and its count in the tiles before
+// this one, the others pass zeros.  `warp_sum` holds kSortBins / 32 words.
+__device__ __forceinline__ void digit_bases(uint32_t total, uint32_t before, uint32_t* warp_sum, uint32_t* base_s) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t inc = total;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    if (tid < kSortBins && lane == 31) warp_sum[warp] = inc;
+    __syncthreads();
+    if (tid < kSortBins) {
+        uint32_t below = 0;
+#pragma unroll
+        for (int w = 0; w < kSortBins / 32; ++w) below += w < warp ? warp_sum[w] : 0u;
+        base_s[tid] = below + (inc - total) + before;
+    }
+    __syncthreads();
+}
+
 // The loss a key came from, where the key says it all; -0/+0 and NaNs (their sign and payload are not in the key) are
 // read back from the table.
 __device__ __forceinline__ float loss_of_key(uint32_t key, const float* __restrict__ losses, int32_t i) {
@@ -519,36 +541,10 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
                 part_bef[q][d] = bef;
             }
             __syncthreads();
-            uint32_t before = 0;
-            if (tid < kSortBins) {
-                before = part_bef[0][tid] + part_bef[1][tid];
-                tot_s[tid] = part_tot[0][tid] + part_tot[1][tid];
+            {
+                const bool mine = tid < kSortBins;
+                digit_bases(mine ? part_tot[0][tid] + part_tot[1][tid] : 0u, mine ? part_bef[0][tid] + part_bef[1][tid] : 0u, tot_s, base_s);
             }
-            __syncthreads();
-            if (warp == 0) {  // exclusive scan of the 512 digit totals, sixteen per lane
-                constexpr int kPer = kSortBins / 32;
-                uint32_t v[kPer], sum = 0;
-#pragma unroll
-                for (int i = 0; i < kPer; ++i) {
-                    v[i] = tot_s[lane * kPer + i];
-                    sum += v[i];
-                }
-                uint32_t inc = sum;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-                    if (lane >= o) inc += n;
-                }
-                uint32_t run = inc - sum;
-#pragma unroll
-                for (int i = 0; i < kPer; ++i) {
-                    tot_s[lane * kPer + i] = run;
-                    run += v[i];
-                }
-            }
-            __syncthreads();
-            if (tid < kSortBins) base_s[tid] = tot_s[tid] + before;
-            __syncthreads();
             const uint32_t first = (tile << tshift) + warp * (R * 32);
 #pragma unroll
             for (int rd = 0; rd < kSortMaxRounds; ++rd) {
@@ -801,41 +797,17 @@ __global__ void __launch_bounds__(kThreads, 1) topk_cluster_kernel(const __grid_
         }
         cluster.sync();
         if (has_tile) {
-            uint32_t before = 0;
-            if (tid < kSortBins) {
-                uint32_t total = 0;
-                for (uint32_t b = 0; b < St; ++b) {
-                    const uint32_t c = mat[b * kSortBins + tid];
-                    total += c;
-                    before += b < rank ? c : 0u;
+            {
+                uint32_t total = 0, before = 0;
+                if (tid < kSortBins) {
+                    for (uint32_t b = 0; b < St; ++b) {
+                        const uint32_t c = mat[b * kSortBins + tid];
+                        total += c;
+                        before += b < rank ? c : 0u;
+                    }
                 }
-                tot_s[tid] = total;
+                digit_bases(total, before, tot_s, base_s);
             }
-            __syncthreads();
-            if (warp == 0) {  // exclusive scan of the 512 digit totals, sixteen per lane
-                constexpr int kPer = kSortBins / 32;
-                uint32_t v[kPer], sum = 0;
-#pragma unroll
-                for (int i = 0; i < kPer; ++i) {
-                    v[i] = tot_s[lane * kPer + i];
-                    sum += v[i];
-                }
-                uint32_t inc = sum;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-                    if (lane >= o) inc += n;
-                }
-                uint32_t run = inc - sum;
-#pragma unroll
-                for (int i = 0; i < kPer; ++i) {
-                    tot_s[lane * kPer + i] = run;
-                    run += v[i];
-                }
-            }
-            __syncthreads();
-            if (tid < kSortBins) base_s[tid] = tot_s[tid] + before;
-            __syncthreads();
 #pragma unroll
             for (int rd = 0; rd < kSortMaxRounds; ++rd) {
                 if (rd < R) {
