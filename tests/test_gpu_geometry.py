@@ -218,3 +218,33 @@ def test_selector_barrier_gives_up_cleanly(L, oracle):
     idx, _ = L.topk_select(v, k, L.ORDER_LOSS_DESC, ws=ws)
     assert L.read_device_status(ws) == 0
     np.testing.assert_array_equal(idx.cpu().numpy(), oracle.topk(h, k, oracle.LOSS_DESC)[0])
+
+
+BOUNDARY_N = [1025, 4095, 4096, 4097, 8191, 8192, 8193, 32_767, 32_768, 32_769, 65_535, 65_536, 65_537, 150_001]
+
+
+@pytest.mark.parametrize("N", BOUNDARY_N)
+def test_selector_at_block_and_tile_boundaries(L, oracle, N):
+    """Pool sizes around the selector's block sizes (4,096 / 8,192 entries, the 65,536-entry limit of the cluster
+    variants) and selection sizes around its sort tiles, on four kinds of tables: loss-like with copies and special
+    values, all equal, strictly increasing, strictly decreasing."""
+    rng = np.random.default_rng(N)
+    tables = {
+        "loss-like": wl.loss_like_vector(N, N, dup_frac=0.03, specials=True),
+        "all equal": np.full(N, 1.25, np.float32),
+        "increasing": np.arange(N, dtype=np.float32),
+        "decreasing": np.arange(N, 0, -1).astype(np.float32),
+    }
+    ks = sorted({1, 2, 1023, 1024, 1025, 2048, 2049, 4096, 4097, 8192, 8193, N // 3, N - 1, N} & set(range(1, N + 1)))
+    ks = [k for k in ks if k <= N]
+    for name, h in tables.items():
+        v = torch.from_numpy(h).cuda()
+        for k in (ks if name == "loss-like" else [ks[int(rng.integers(len(ks)))], N]):
+            for order in (L.ORDER_LOSS_DESC, L.ORDER_INDEX_ASC):
+                want_idx, want_vals = oracle.topk(h, k, order)
+                for kw in (dict(), dict(narrow_cluster=True)) if N <= 65_536 else (dict(),):
+                    with geometry(**kw):
+                        idx, vals = L.topk_select(v, k, order)
+                    np.testing.assert_array_equal(idx.cpu().numpy(), want_idx, err_msg=f"{name} N={N} k={k} order={order} {kw}")
+                    np.testing.assert_array_equal(vals.cpu().numpy().view(np.uint32), want_vals.view(np.uint32),
+                                                  err_msg=f"{name} N={N} k={k} order={order} {kw}")
