@@ -18,8 +18,7 @@
 //   small rows  (<= 2 KB)                        4, 8 or 16 lanes per row out of a block's shared-memory tile
 //   medium rows (<= 256 KB)                      one warp per row, streamed through registers with a running (max, sum)
 //   anything longer                              one CTA per row, two passes over global memory
-// (a pool whose base is not 16-byte aligned takes the lane-group kernel or, for rows of at most 32 elements, a
-// thread-per-row kernel with element-wise staging).
+// (rows of 417 bytes to 2 KB of a pool whose base is not 16-byte aligned are read element by element from the tile).
 // Rows whose label is ignore_index are never scored; the kernels for medium and longer rows do not even
 // read them (short and small rows are copied block-wise, ignored rows included).
 #include <cuda_bf16.h>
@@ -225,70 +224,7 @@ __device__ __forceinline__ void cp_async_wait() {
 }
 
 // ---------------------------------------------------------------------------
-// Tiny rows with a pool base that is not 16-byte aligned: a CTA stages 256
-// consecutive rows (contiguous in memory) into shared memory with coalesced
-// element loads; each thread then owns one row.
-// ---------------------------------------------------------------------------
-
-template <typename T>
-__global__ void __launch_bounds__(kTinyThreads)
-score_tiny_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
-                       int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0) {
-    __shared__ float tile[kTinyThreads * (kTinyMaxC + 1)];
-    __shared__ uint32_t hist_s[kSelBins];
-    Hist0 h{hist_s, hist0};
-    h.clear();
-    const int pitch = C | 1;  // odd pitch: conflict-free row reads
-    const int step_r = kTinyThreads / C, step_c = kTinyThreads - step_r * C;
-    const int64_t tiles = (rows + kTinyThreads - 1) / kTinyThreads;
-    for (int64_t t = blockIdx.x; t < tiles; t += gridDim.x) {
-        const int64_t row0 = t * kTinyThreads;
-        const int nrows = rows - row0 < kTinyThreads ? static_cast<int>(rows - row0) : kTinyThreads;
-        const T* src = logits + row0 * C;
-        const int n = nrows * C;
-        __syncthreads();
-        {   // element i = r C + c; i advances by the CTA size, (r, c) by its quotient and remainder
-            int r = threadIdx.x / C, c = threadIdx.x - r * C;
-            for (int i = threadIdx.x; i < n; i += kTinyThreads) {
-                tile[r * pitch + c] = Elem<T>::widen(src[i]);
-                r += step_r;
-                c += step_c;
-                if (c >= C) {
-                    c -= C;
-                    ++r;
-                }
-            }
-        }
-        __syncthreads();
-        if (threadIdx.x < nrows) {
-            const int64_t row = row0 + threadIdx.x;
-            const int64_t y = labels[row];
-            const int cls = label_class(y, C, ignore_index);
-            float loss = 0.f;
-            if (cls == 2) {
-                loss = __uint_as_float(0x7FC00000u);
-                atomicAdd(&status->bad_labels, 1);
-            } else if (cls == 0) {
-                float* x = tile + threadIdx.x * pitch;
-                const float xy = x[static_cast<int>(y)];
-                x[static_cast<int>(y)] = neg_inf();  // the true class stays out of the sum
-                float m = -1e30f;
-                for (int j = 0; j < C; ++j) m = fmaxf(m, x[j]);
-                const float P = m * kLog2e;
-                float s = 0.f;
-                for (int j = 0; j < C; ++j) s += ex2(fmaf(x[j], kLog2e, -P));
-                loss = loss_without_true_class(m, P, s, xy);
-            }
-            row_loss[row] = loss;
-            h.add(loss);
-        }
-    }
-    __syncthreads();
-    h.flush();
-}
-
-// ---------------------------------------------------------------------------
-// Small rows (417 bytes to 2 KB; shorter ones of an unaligned pool): a CTA copies a tile of consecutive rows (one
+// Small rows (417 bytes to 2 KB): a CTA copies a tile of consecutive rows (one
 // contiguous, 16-byte-aligned-superset byte range) into shared memory with
 // vector loads; groups of L lanes then own one row each and read it from there.
 // One warp per row would spend most of its instructions on 32-lane reductions
@@ -558,13 +494,14 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
 }
 
 // ---------------------------------------------------------------------------
-// Short rows (up to kLaneMaxRowBytes), pool base 16-byte aligned: a WARP takes 32 consecutive rows (one
-// contiguous, 16-byte aligned byte range), brings them into its own ring of shared-memory stages with 16-byte
-// asynchronous copies, one or two blocks of rows ahead of the one being scored, and every LANE scores one row.
+// Short rows (up to kLaneMaxRowBytes, or at most 32 elements): a WARP takes 32 consecutive rows (one contiguous
+// byte range; 32 rows are a multiple of 16 bytes, so every block starts at the same offset `head` from a 16-byte
+// boundary), brings their aligned superset into its own ring of shared-memory stages with 16-byte asynchronous copies, one or two blocks of rows ahead of the one being scored, and every LANE scores one row.
 // Nothing in the loop synchronises more than a warp, and the per-row work (label, reductions, the logarithm) is
-// done once per lane instead of once per group of lanes.  Rows that are whole 16-byte chunks are laid out at an
-// odd chunk pitch; other rows are copied flat and read in units of the largest power of two (8, 4 or 2 bytes) that
-// divides the row length, so that the lanes' strides are odd multiples of the unit: no bank conflicts either way.
+// done once per lane instead of once per group of lanes.  Rows that are whole 16-byte chunks (of an aligned pool)
+// are laid out at an odd chunk pitch; other rows are copied flat and read in units of the largest power of two (8, 4
+// or 2 bytes) that divides the row length and the offset `head`, so that the lanes' strides are odd multiples of the
+// unit: no bank conflicts either way (except for whole-chunk rows of a misaligned pool, which are merely correct).
 // CMAX > 0 (rows of at most 32 elements): the row is read once into CMAX registers (slots past C hold -inf).
 // CMAX == 0: two passes over the row in shared memory (maximum, then the sum), in units of CB bytes.
 // A row's sum runs over its elements in an order that depends on C only, so copies of a row score the same bits
@@ -577,8 +514,8 @@ template <typename T, int CMAX, int CB, int STAGES>
 __global__ void __launch_bounds__(CMAX > 0 ? kTinyThreads : kLaneThreads)
 score_lane_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
                        int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0,
-                       int stage_bytes) {
-    constexpr bool PADDED = CB == 16;
+                       int stage_bytes, int head) {
+    constexpr bool PADDED = CB == 16;  // (only with head == 0)
     constexpr int kWarpsPerCta = (CMAX > 0 ? kTinyThreads : kLaneThreads) / 32;
     extern __shared__ __align__(16) unsigned char lane_smem[];
     uint32_t* hist_s = reinterpret_cast<uint32_t*>(lane_smem);
@@ -609,15 +546,12 @@ score_lane_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
         if (i < mine) {
             const int64_t row0 = (gw + i * nw) << 5;
             const int nrows = rows - row0 < 32 ? static_cast<int>(rows - row0) : 32;
-            const unsigned char* src = reinterpret_cast<const unsigned char*>(logits) + row0 * row_bytes;
+            // the 16-byte-aligned superset of the block's bytes (every block starts `head` bytes past a boundary;
+            // an aligned 16-byte unit that holds one valid byte is safe to read in full)
+            const unsigned char* src = reinterpret_cast<const unsigned char*>(logits) + row0 * row_bytes - head;
             unsigned char* dst = ring + (i % STAGES) * stage_bytes;
-            const int bytes = nrows * row_bytes, nvec = bytes >> 4;
+            const int nvec = (head + nrows * row_bytes + 15) >> 4;
             for (int v = lane; v < nvec; v += 32) cp_async16(dst + place(v) * 16, src + v * 16);
-            // a last, partial chunk (only at the very end of the pool) is copied element by element
-            for (int e = (nvec << 4) / ES + lane; e < bytes / ES; e += 32) {
-                const int byte = e * ES;
-                *reinterpret_cast<T*>(dst + place(byte >> 4) * 16 + (byte & 15)) = reinterpret_cast<const T*>(src)[e];
-            }
             if (lane < nrows) y = labels[row0 + lane];
         }
         cp_async_commit();  // one group per slot, also when it is empty: the wait below counts groups
@@ -642,7 +576,7 @@ score_lane_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
         const bool valid = row0 + lane < rows;
         unsigned char* buf = ring + (i % STAGES) * stage_bytes;
         const int cls = valid ? label_class(y, C, ignore_index) : 1;
-        T* rowe = reinterpret_cast<T*>(buf + (PADDED ? lane * pitch * 16 : lane * row_bytes));
+        T* rowe = reinterpret_cast<T*>(buf + (PADDED ? lane * pitch * 16 : head + lane * row_bytes));
         // the true class stays out of the sum (see loss_without_true_class): its slot is read, then blanked
         float xy = 0.f;
         if (cls == 0) {
@@ -996,14 +930,16 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
     const int sms = sm_count();
     const int64_t max_ctas = test_geometry().max_ctas;
     const int64_t row_bytes = C * static_cast<int64_t>(sizeof(T));
-    const bool base16 = (reinterpret_cast<uintptr_t>(logits) & 15) == 0;
-    if (base16 && (C <= kTinyMaxC || row_bytes <= kLaneMaxRowBytes)) {
+    if (C <= kTinyMaxC || row_bytes <= kLaneMaxRowBytes) {
         // one lane per row: the access unit is the largest power of two (at most 16 bytes) that divides the row
+        // length and the pool's offset from a 16-byte boundary
         cudaError_t err = cudaSuccess;
-        const int cb = row_bytes % 16 == 0 ? 16 : row_bytes % 8 == 0 ? 8 : row_bytes % 4 == 0 ? 4 : 2;
+        const int head = static_cast<int>(reinterpret_cast<uintptr_t>(logits) & 15);
+        const int64_t both = row_bytes | head;
+        const int cb = both % 16 == 0 ? 16 : both % 8 == 0 ? 8 : both % 4 == 0 ? 4 : 2;
         auto go = [&](auto kernel, int threads, int stages) {
             const int64_t rc = row_bytes / 16;
-            const int stage_bytes = static_cast<int>(cb == 16 ? 32 * (rc | 1) * 16 : (32 * row_bytes + 15) / 16 * 16);
+            const int stage_bytes = static_cast<int>(cb == 16 ? 32 * (rc | 1) * 16 : (head + 32 * row_bytes + 15) / 16 * 16);
             const size_t smem = (hist0 ? kSelBins * sizeof(uint32_t) : 0) + static_cast<size_t>(threads / 32) * stages * stage_bytes;
             const int bps = blocks_per_sm(kernel, threads, smem, true);
             if (bps < 1) {
@@ -1013,7 +949,7 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
             const int64_t want = ((rows + 31) / 32 + threads / 32 - 1) / (threads / 32);
             const int grid = static_cast<int>(std::min({want, static_cast<int64_t>(sms) * bps, max_ctas}));
             kernel<<<grid, threads, smem, s>>>(logits, labels, rows, static_cast<int>(C), ignore_index, row_loss, status,
-                                               hist0, stage_bytes);
+                                               hist0, stage_bytes, head);
             err = cudaGetLastError();
         };
         if (C <= kTinyMaxC) {
@@ -1041,7 +977,7 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
         // A pool so small that, with a single stage per warp, every block of 32 rows gets a warp of its own at once:
         // nothing to pipeline, and twice the warps are resident (a CIFAR-sized pool is scored in one wave).
         {
-            const int64_t stage1 = cb == 16 ? 32 * ((row_bytes / 16) | 1) * 16 : (32 * row_bytes + 15) / 16 * 16;
+            const int64_t stage1 = cb == 16 ? 32 * ((row_bytes / 16) | 1) * 16 : (head + 32 * row_bytes + 15) / 16 * 16;
             const int64_t per_cta = (hist0 ? kSelBins * sizeof(uint32_t) : 0) + (kLaneThreads / 32) * stage1 + 1024;
             const int64_t ctas = std::min<int64_t>(32, (227 * 1024) / per_cta);
             if ((rows + 31) / 32 <= static_cast<int64_t>(sms) * ctas * (kLaneThreads / 32) && max_ctas >= static_cast<int64_t>(sms) * ctas) {
@@ -1054,13 +990,6 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
         if (32 * row_bytes <= 4608) by_unit(std::integral_constant<int, 3>{});
         else by_unit(std::integral_constant<int, 2>{});
         return err;
-    }
-    if (C <= kTinyMaxC) {
-        const int64_t tiles = (rows + kTinyThreads - 1) / kTinyThreads;
-        const int grid = static_cast<int>(std::min({tiles, static_cast<int64_t>(sms) * 8, max_ctas}));
-        score_tiny_rows_kernel<T><<<grid, kTinyThreads, 0, s>>>(logits, labels, rows, static_cast<int>(C),
-                                                                 ignore_index, row_loss, status, hist0);
-        return cudaGetLastError();
     }
     if (row_bytes <= kGroupMaxRowBytes) {
         const bool base_ok = (reinterpret_cast<uintptr_t>(logits) & 15) == 0;

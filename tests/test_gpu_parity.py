@@ -81,11 +81,12 @@ def test_score_matches_oracle(L, oracle, N, T, C, dtype):
     assert_losses_close(got.cpu().numpy(), want, C)
 
 
-@pytest.mark.parametrize("C,dtype", [(10, "f32"), (100, "f32"), (1000, "bf16"), (5000, "f32"), (30522, "bf16")])
-@pytest.mark.parametrize("off", [1, 2, 3])
+@pytest.mark.parametrize("C,dtype", [(10, "f32"), (7, "bf16"), (32, "f32"), (32, "bf16"), (100, "f32"), (100, "bf16"), (101, "bf16"), (104, "f32"),
+                                     (300, "bf16"), (1000, "bf16"), (5000, "f32"), (30522, "bf16")])
+@pytest.mark.parametrize("off", [1, 2, 3, 4, 5])
 def test_score_misaligned_base(L, oracle, C, dtype, off):
     # the pool starts `off` elements into an allocation: rows start at every 4-byte (2-byte) phase
-    N = 41
+    N = 41 if C > 1000 else 777
     x, y = random_pool(7, N, 1, C, dtype)
     flat = dev_logits(x).reshape(-1)
     buf = torch.zeros(flat.numel() + 8, dtype=flat.dtype, device="cuda")
