@@ -229,9 +229,10 @@ __device__ __forceinline__ void cp_async_wait() {
 // vector loads; groups of L lanes then own one row each and read it from there.
 // One warp per row would spend most of its instructions on 32-lane reductions
 // and on the per-row epilogue; with L lanes per row those are shared by 32 / L
-// rows.  With a 16-byte-aligned base, rows start on 16-, 8- or 4-byte boundaries
-// according to their length, and a lane reads chunks of that size, l, l + L, ...
-// of its row; otherwise it reads elements l, l + L, ...
+// rows.  Rows start on 16-, 8- or 4-byte boundaries according to their length and
+// to the pool's offset from a 16-byte boundary (every tile starts at that offset),
+// and a lane reads chunks of that size, l, l + L, ... of its row; rows that start on
+// odd 2-byte boundaries are read element by element.
 // ---------------------------------------------------------------------------
 constexpr int kGroupThreads = 128;
 constexpr int kGroupMaxRowBytes = 2048;
@@ -347,7 +348,7 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
                         int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0,
                         int stage_bytes) {
     constexpr int R = kGroupThreads / L;  // rows per tile = lane groups per CTA
-    constexpr bool VEC = CB > 0;          // rows start on CB-byte boundaries and are whole chunks (base 16-byte aligned)
+    constexpr bool VEC = CB > 0;          // rows start on CB-byte boundaries and are whole chunks
     constexpr bool PADDED = CB == 16 && L < 8;
     extern __shared__ __align__(16) unsigned char group_smem[];
     unsigned char* stages = group_smem;
@@ -370,7 +371,7 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
             const int64_t row0 = (blockIdx.x + i * gridDim.x) * R;
             const int nrows = rows - row0 < R ? static_cast<int>(rows - row0) : R;
             const uintptr_t b0 = reinterpret_cast<uintptr_t>(logits) + row0 * row_bytes;
-            const int head = VEC ? 0 : static_cast<int>(b0 & 15);
+            const int head = static_cast<int>(b0 & 15);  // the same for every tile: a tile's rows are a multiple of 16 bytes
             const uint4* src = reinterpret_cast<const uint4*>(b0 - head);
             const int nvec = (head + nrows * row_bytes + 15) >> 4;  // an aligned block that holds a valid byte is safe to read
             uint4* dst = reinterpret_cast<uint4*>(stages + (i % kGroupStages) * stage_bytes);
@@ -401,7 +402,7 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
         __syncthreads();  // everybody's copies of tile i have landed
         const int64_t row0 = (blockIdx.x + i * gridDim.x) * R;
         const bool mine = row0 + g < rows;
-        const int head = VEC ? 0 : static_cast<int>((reinterpret_cast<uintptr_t>(logits) + row0 * row_bytes) & 15);
+        const int head = static_cast<int>((reinterpret_cast<uintptr_t>(logits) + row0 * row_bytes) & 15);
         unsigned char* buf = stages + (i % kGroupStages) * stage_bytes;
         const int cls = mine ? label_class(y, C, ignore_index) : 1;
         T* x = reinterpret_cast<T*>(buf + head + g * pitch_bytes);
@@ -992,8 +993,10 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
         return err;
     }
     if (row_bytes <= kGroupMaxRowBytes) {
-        const bool base_ok = (reinterpret_cast<uintptr_t>(logits) & 15) == 0;
-        const int cb = !base_ok ? 0 : row_bytes % 16 == 0 ? 16 : row_bytes % 8 == 0 ? 8 : row_bytes % 4 == 0 ? 4 : 0;
+        // the unit a lane reads: the largest power of two that divides the row length and the pool's offset from a
+        // 16-byte boundary (every tile starts at that offset), 0 = single elements
+        const int64_t both = row_bytes | static_cast<int64_t>(reinterpret_cast<uintptr_t>(logits) & 15);
+        const int cb = both % 16 == 0 ? 16 : both % 8 == 0 ? 8 : both % 4 == 0 ? 4 : 0;
         cudaError_t err = cudaSuccess;
         auto go = [&](auto kernel, int lanes) {
             const int tile_rows = kGroupThreads / lanes;
