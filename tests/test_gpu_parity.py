@@ -409,3 +409,34 @@ def test_errors_raise(L):
         L.aggregate([torch.zeros(8, device="cuda")] * 65, [0.0] * 65)
     # a failed call leaves the context usable
     assert L.score_losses(x, y).shape == (4,)
+
+
+def test_score_random_shapes_offsets_and_masks(L, oracle):
+    """A seeded sweep over row lengths of every kernel's range, both types, pools starting at every element offset
+    inside an allocation, ignored and out-of-range labels: every loss against the oracle."""
+    rng = np.random.default_rng(20250808)
+    lengths = list(range(1, 40)) + [rng.integers(40, 210) for _ in range(40)] + [rng.integers(210, 1100) for _ in range(25)] + \
+              [int(x) for x in rng.integers(1100, 9000, 8)]
+    for case, C in enumerate(lengths):
+        C = int(C)
+        dtype = "bf16" if case % 2 else "f32"
+        N = int(rng.integers(1, 400 if C < 1100 else 60))
+        T = 1 if case % 5 else 3
+        off = int(rng.integers(0, 8))
+        x, y = random_pool(1000 + case, N, T, C, dtype, sigma=float(rng.choice([0.5, 2.0, 8.0])), bump=float(rng.choice([0.0, 3.0])),
+                           mask_p=0.2 if T > 1 else 0.0)
+        y = y.copy()
+        if case % 7 == 0:
+            y.reshape(-1)[rng.integers(0, y.size)] = C + 5  # one label out of range
+        flat = dev_logits(x).reshape(-1)
+        buf = torch.zeros(flat.numel() + 8, dtype=flat.dtype, device="cuda")
+        buf[off:off + flat.numel()] = flat
+        view = buf[off:off + flat.numel()].view(N, T, C)
+        want, bad = oracle.score(x, y)
+        ws = L.workspace(L.score_workspace_bytes(N, T, C))
+        got = L.score_losses(view, torch.from_numpy(y).cuda(), ws=ws).cpu().numpy()
+        assert L.read_device_status(ws) == bad, (case, C, dtype, N, T, off)
+        nan = np.isnan(want)
+        assert np.array_equal(np.isnan(got), nan), (case, C, dtype, N, T, off)
+        err = np.abs(got[~nan].astype(np.float64) - want[~nan])
+        assert (err <= 1e-5 * np.abs(want[~nan]) + C * 2.0 ** -52).all(), (case, C, dtype, N, T, off, float(err.max()))
