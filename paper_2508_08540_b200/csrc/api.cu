@@ -141,8 +141,7 @@ lsgd_status lsgd_topk_select(const float* losses, int64_t N, int64_t k, lsgd_ord
     st = check_ws(ws, ws_bytes, topk_workspace_bytes(N, k));
     if (st != LSGD_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    if (zero_topk_workspace(ws, k, s) != cudaSuccess) return LSGD_ERR_CUDA;
-    return from_cuda(launch_topk(losses, N, k, order, out_idx, out_vals, carve_topk(ws, N, k), false, s));
+    return from_cuda(launch_topk(losses, N, k, order, out_idx, out_vals, carve_topk(ws, N, k), false, true, s));
 }
 
 lsgd_status lsgd_score_topk(const void* logits, lsgd_dtype dtype, const int64_t* labels, int64_t N, int64_t T,
@@ -169,7 +168,7 @@ lsgd_status lsgd_score_topk(const void* logits, lsgd_dtype dtype, const int64_t*
                                  fuse_hist ? tw.hist : nullptr, s);
     if (e != cudaSuccess) return LSGD_ERR_CUDA;
     if (k == 0) return LSGD_OK;
-    return from_cuda(launch_topk(losses, N, k, order, out_idx, out_vals, tw, fuse_hist, s));
+    return from_cuda(launch_topk(losses, N, k, order, out_idx, out_vals, tw, fuse_hist, false, s));
 }
 
 lsgd_status lsgd_aggregate(const float* const* replicas, const float* weights, int32_t P, int64_t D, float* out,

@@ -72,7 +72,8 @@ size_t topk_workspace_bytes(int64_t N, int64_t k);
 size_t score_workspace_bytes(int64_t N, int64_t T, int64_t C);
 TopkWorkspace carve_topk(void* ws, int64_t N, int64_t k);
 ScoreWorkspace carve_score(void* ws, int64_t N, int64_t T, int64_t C);
-// Clears the status block, the selector's histograms and the sort's digit counts.
+// Clears the status block and the selector's histograms.  The fused call does this before the scorer runs; a
+// selection on its own (launch_topk with `standalone`) clears whatever its kernel needs itself.
 cudaError_t zero_topk_workspace(void* ws, int64_t k, cudaStream_t s);
 
 // Launchers (each returns the CUDA error of its launches).  `hist0` non-NULL asks
@@ -84,7 +85,7 @@ cudaError_t launch_score(const void* logits, lsgd_dtype dt, const int64_t* label
                          int64_t ignore_index, float* losses, const ScoreWorkspace& ws, uint32_t* hist0,
                          cudaStream_t s);
 cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order order, int32_t* out_idx,
-                        float* out_vals, const TopkWorkspace& ws, bool hist0_ready, cudaStream_t s);
+                        float* out_vals, const TopkWorkspace& ws, bool hist0_ready, bool standalone, cudaStream_t s);
 
 int sm_count();  // multiprocessors of the current device (cached per device)
 

@@ -101,8 +101,7 @@ lsgd_status check_ws(const void* ws, size_t have, size_t need) {
 cudaError_t enqueue_draw(int64_t N, int64_t m, uint64_t seed, uint64_t stream, const int32_t* exclude_idx,
                          int64_t n_exclude, int32_t* out_idx, void* ws, size_t sel_bytes, cudaStream_t s) {
     float* pri = reinterpret_cast<float*>(static_cast<unsigned char*>(ws) + sel_bytes);
-    cudaError_t e = zero_topk_workspace(ws, m, s);
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
     priority_kernel<<<grid_for((N + 3) / 4), kThreads, 0, s>>>(pri, N, static_cast<uint32_t>(seed),
                                                                static_cast<uint32_t>(seed >> 32),
                                                                static_cast<uint32_t>(stream),
@@ -110,7 +109,7 @@ cudaError_t enqueue_draw(int64_t N, int64_t m, uint64_t seed, uint64_t stream, c
     if (n_exclude > 0) exclude_kernel<<<grid_for(n_exclude), kThreads, 0, s>>>(pri, N, exclude_idx, n_exclude);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    return launch_topk(pri, N, m, LSGD_ORDER_LOSS_DESC, out_idx, nullptr, carve_topk(ws, N, m), false, s);
+    return launch_topk(pri, N, m, LSGD_ORDER_LOSS_DESC, out_idx, nullptr, carve_topk(ws, N, m), false, true, s);
 }
 
 }  // namespace
@@ -184,8 +183,7 @@ lsgd_status lsgd_fast_allocation(const float* losses, int64_t N, int64_t k_high,
     if (st != LSGD_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     if (k_high > 0) {
-        if (zero_topk_workspace(ws, k_high, s) != cudaSuccess) return LSGD_ERR_CUDA;
-        if (launch_topk(losses, N, k_high, LSGD_ORDER_LOSS_DESC, out_idx, nullptr, carve_topk(ws, N, k_high), false, s) !=
+        if (launch_topk(losses, N, k_high, LSGD_ORDER_LOSS_DESC, out_idx, nullptr, carve_topk(ws, N, k_high), false, true, s) !=
             cudaSuccess)
             return LSGD_ERR_CUDA;
     }

@@ -71,10 +71,9 @@ extern "C" lsgd_status lsgd_topk_select_static(const float* losses, int64_t N, i
     void* ws = scratch_on_current_device();
     if (!ws) return LSGD_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    // the array keeps whatever the previous call left: status block, histograms and digit
-    // counts must start at zero
-    if (zero_topk_workspace(ws, k, s) != cudaSuccess) return LSGD_ERR_CUDA;
-    return launch_topk(losses, N, k, order, out_idx, out_vals, carve_topk(ws, N, k), false, s) == cudaSuccess
+    // the array keeps whatever the previous call left: the launcher clears what its kernel needs to start at zero
+    // (the status block and the digit histograms)
+    return launch_topk(losses, N, k, order, out_idx, out_vals, carve_topk(ws, N, k), false, true, s) == cudaSuccess
                ? LSGD_OK
                : LSGD_ERR_CUDA;
 }

@@ -114,6 +114,7 @@ struct SelectParams {
     int hist0_ready;      // the first digit's histogram was accumulated by the scorer
     uint32_t barrier_parties;  // blocks a barrier waits for: gridDim.x (a test hook adds one that never arrives)
     uint32_t barrier_polls;    // polls after which a block gives up
+    int standalone;            // a selection on its own (no scorer before it in the call): the kernel resets the status block
 };
 
 __device__ __forceinline__ uint32_t digit_of(uint32_t key, int pass) {
@@ -619,6 +620,10 @@ __global__ void __launch_bounds__(kThreads, 1) topk_cluster_kernel(const __grid_
     cluster.sync();          // every block's accumulators are clear before anybody adds to them
     grid_dependency_wait();  // the losses (and the scorer's histogram) are complete from here on
 
+    if (p.standalone && rank == 0 && tid == 0) {  // a selection on its own: the status block reads "nothing to report"
+        p.ws.status->bad_labels = 0;
+        p.ws.status->timeout = 0;
+    }
     uint32_t key[kClE];
     load_keys<kClE>(losses, N, static_cast<int64_t>(rank) * kClTile + static_cast<int64_t>(tid) * kClE, key);
 
@@ -835,10 +840,14 @@ constexpr int kSmallThreads = 1024;
 
 __global__ void __launch_bounds__(kSmallThreads)
 small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int32_t* __restrict__ out_idx,
-                  float* __restrict__ out_vals) {
+                  float* __restrict__ out_vals, StatusBlock* status) {
     __shared__ unsigned long long ck[kSmallN];
     __shared__ uint32_t warp_tot[kSmallThreads / 32];
     grid_dependency_wait();
+    if (status && threadIdx.x == 0) {  // a selection on its own: the status block reads "nothing to report"
+        status->bad_labels = 0;
+        status->timeout = 0;
+    }
     int n2 = 1;
     while (n2 < n) n2 <<= 1;
     for (int i = threadIdx.x; i < n2; i += kSmallThreads)
@@ -1019,10 +1028,10 @@ int resident_blocks() {
 }  // namespace
 
 cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order order, int32_t* out_idx,
-                        float* out_vals, const TopkWorkspace& ws, bool hist0_ready, cudaStream_t s) {
+                        float* out_vals, const TopkWorkspace& ws, bool hist0_ready, bool standalone, cudaStream_t s) {
     if (N <= kSmallN)
         return launch_dependent(small_topk_kernel, 1, kSmallThreads, s, losses, static_cast<int>(N), static_cast<int>(k),
-                                static_cast<int>(order), out_idx, out_vals);
+                                static_cast<int>(order), out_idx, out_vals, standalone ? ws.status : nullptr);
     SelectParams p;
     p.losses = losses;
     p.N = N;
@@ -1032,6 +1041,7 @@ cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order or
     p.out_vals = out_vals;
     p.ws = ws;
     p.hist0_ready = hist0_ready ? 1 : 0;
+    p.standalone = standalone ? 1 : 0;
     p.barrier_parties = 0;
     p.barrier_polls = kMaxPolls;
     const TestGeometry tg = test_geometry();
@@ -1046,6 +1056,11 @@ cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order or
             p.sort_tiles = static_cast<uint32_t>((k + 1024 * p.sort_rounds - 1) / (1024 * p.sort_rounds));
             return wide ? launch_cluster<4, 16>(p, grid, s) : launch_cluster<8, 8>(p, grid, s);
         }
+    }
+    // the cooperative kernel accumulates histograms in the workspace and counts barrier arrivals in the status block
+    if (standalone) {
+        const cudaError_t ze = zero_topk_workspace(ws.status, k, s);
+        if (ze != cudaSuccess) return ze;
     }
     const int resident = std::max(1, std::min(resident_blocks(), tg.max_ctas));
     p.sort_rounds = sort_rounds_for(k, std::min(resident, kSortDirectTiles));

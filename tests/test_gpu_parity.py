@@ -440,3 +440,26 @@ def test_score_random_shapes_offsets_and_masks(L, oracle):
         assert np.array_equal(np.isnan(got), nan), (case, C, dtype, N, T, off)
         err = np.abs(got[~nan].astype(np.float64) - want[~nan])
         assert (err <= 1e-5 * np.abs(want[~nan]) + C * 2.0 ** -52).all(), (case, C, dtype, N, T, off, float(err.max()))
+
+
+@pytest.mark.parametrize("N", [500, 5_000, 100_000])
+def test_fused_call_reports_bad_labels_and_a_selection_alone_reports_none(L, oracle, N):
+    """The status block after lsgd_score_topk carries the scorer's count through every selector variant (one block,
+    one cluster, cooperative); after a selection on its own it reads zero, whatever the workspace held before."""
+    C = 10
+    x, y = random_pool(5, N, 1, C, "f32")
+    y = y.copy()
+    y[[1, N // 2, N - 1]] = C + 1
+    xd, yd = dev_logits(x), torch.from_numpy(y).cuda()
+    k = N // 4
+    ws = L.workspace(L.score_topk_workspace_bytes(N, 1, C, k))
+    ws.fill_(0xFF)
+    losses, idx, _ = L.score_topk(xd, yd, k, L.ORDER_LOSS_DESC, ws=ws)
+    assert L.read_device_status(ws) == 3
+    g = losses.cpu().numpy()
+    assert np.isnan(g).sum() == 3
+    np.testing.assert_array_equal(idx.cpu().numpy(), oracle.topk(g, k, oracle.LOSS_DESC)[0])  # NaN ranks highest
+    ws.fill_(0xFF)
+    idx2, _ = L.topk_select(losses, k, L.ORDER_LOSS_DESC, ws=ws)
+    assert L.read_device_status(ws) == 0
+    assert torch.equal(idx, idx2)
