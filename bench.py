@@ -496,7 +496,7 @@ def launches_per_step(cfg) -> int:
     """Kernels of liblsgd launched by one step (memsets excluded), from the launch logic of the library."""
     n = 1 + (1 if cfg.T > 1 else 0)                # scorer (+ sequence mean)
     n += 1                                          # the selector is one kernel at every pool size
-    n += 1 + (1 if cfg.D % 4 else 0)                # aggregation (+ ragged tail)
+    n += 1                                          # aggregation
     return n
 
 

@@ -39,7 +39,14 @@ __device__ __forceinline__ float4 mul4(float w, float4 v) { return make_float4(w
 // `out` carries no no-alias promise: it may be one of the replicas (in-place update).
 template <int PCT>
 __global__ void __launch_bounds__(kAggThreads) aggregate_vec4_kernel(const __grid_constant__ AggArgs a, int P,
-                                                                      int64_t n4, float* out) {
+                                                                      int64_t n4, int64_t D, float* out) {
+    // the up to three elements past the last whole slice: one thread each, same chain of operations
+    if (blockIdx.x == 0 && 4 * n4 + threadIdx.x < D) {
+        const int64_t j = 4 * n4 + threadIdx.x;
+        float acc = a.w[0] * __ldcg(a.x[0] + j);
+        for (int r = 1; r < P; ++r) acc = fmaf(a.w[r], __ldcg(a.x[r] + j), acc);
+        out[j] = acc;
+    }
     const int64_t stride = static_cast<int64_t>(gridDim.x) * kAggThreads;
     for (int64_t i = static_cast<int64_t>(blockIdx.x) * kAggThreads + threadIdx.x; i < n4; i += stride) {
         float4 acc;
@@ -66,8 +73,7 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_vec4_kernel(const __gri
     }
 }
 
-// Scalar path: the ragged tail of the vector path (elements [begin, D)), and the
-// whole vector when some pointer is not 16-byte aligned.
+// Scalar path: the whole vector when some pointer is not 16-byte aligned (or D < 4).
 __global__ void __launch_bounds__(kAggThreads) aggregate_scalar_kernel(const __grid_constant__ AggArgs a, int P,
                                                                         int64_t begin, int64_t D,
                                                                         float* out) {
@@ -80,7 +86,7 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_scalar_kernel(const __g
 }
 
 template <int PCT>
-cudaError_t launch_vec(const AggArgs& a, int P, int64_t n4, float* out, cudaStream_t s) {
+cudaError_t launch_vec(const AggArgs& a, int P, int64_t n4, int64_t D, float* out, cudaStream_t s) {
     static int blocks_per_sm[64] = {0};
     int dev = 0;
     cudaGetDevice(&dev);
@@ -94,7 +100,7 @@ cudaError_t launch_vec(const AggArgs& a, int P, int64_t n4, float* out, cudaStre
     const int64_t want = (n4 + kAggThreads - 1) / kAggThreads;
     const int64_t cap = static_cast<int64_t>(sm_count()) * bps;
     const int grid = static_cast<int>(want < cap ? want : cap);
-    aggregate_vec4_kernel<PCT><<<grid, kAggThreads, 0, s>>>(a, P, n4, out);
+    aggregate_vec4_kernel<PCT><<<grid, kAggThreads, 0, s>>>(a, P, n4, D, out);
     return cudaGetLastError();
 }
 
@@ -113,18 +119,18 @@ cudaError_t launch_aggregate(const float* const* replicas, const float* weights,
         switch (P) {
 #define LSGD_AGG_CASE(n) \
     case n:              \
-        e = launch_vec<n>(a, P, n4, out, s); \
+        e = launch_vec<n>(a, P, n4, D, out, s); \
         break;
             LSGD_AGG_CASE(1) LSGD_AGG_CASE(2) LSGD_AGG_CASE(3) LSGD_AGG_CASE(4) LSGD_AGG_CASE(5) LSGD_AGG_CASE(6)
             LSGD_AGG_CASE(7) LSGD_AGG_CASE(8) LSGD_AGG_CASE(9) LSGD_AGG_CASE(10) LSGD_AGG_CASE(11)
             LSGD_AGG_CASE(12) LSGD_AGG_CASE(13) LSGD_AGG_CASE(14) LSGD_AGG_CASE(15) LSGD_AGG_CASE(16)
 #undef LSGD_AGG_CASE
             default:
-                e = launch_vec<0>(a, P, n4, out, s);
+                e = launch_vec<0>(a, P, n4, D, out, s);
         }
         if (e != cudaSuccess) return e;
     }
-    const int64_t begin = n4 * 4;
+    const int64_t begin = n4 > 0 ? D : 0;  // the vector kernel takes its own ragged tail along
     if (begin < D) {
         const int64_t rest = D - begin;
         const int64_t want = (rest + kAggThreads - 1) / kAggThreads;
