@@ -452,14 +452,14 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
             using Word = typename ChunkWord<VEC ? CB : 16>::type;
             const Word* xv = reinterpret_cast<const Word*>(x);
             const int nch = cls == 0 ? nchunk : 0;
-#pragma unroll 2
+#pragma unroll 4
             for (int c = l; c < nch; c += L) m = fmaxf(m, chunk_max<T, VEC ? CB : 16>(xv[c]));
 #pragma unroll
             for (int o = L / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
             const float P = m * kLog2e;
             const F2 l2e = pack2(kLog2e, kLog2e), nml = pack2(-P, -P);
             F2 a0 = pack2(0.f, 0.f), a1 = pack2(0.f, 0.f);
-#pragma unroll 2
+#pragma unroll 4
             for (int c = l; c < nch; c += L) chunk_sum_exp<T, VEC ? CB : 16>(xv[c], l2e, nml, a0, a1);
             float t0, t1, t2, t3;
             unpack2(a0, t0, t1);
