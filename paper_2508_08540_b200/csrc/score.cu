@@ -342,7 +342,9 @@ __device__ __forceinline__ void chunk_sum_exp(const typename ChunkWord<CB>::type
 // Tiles flow through a ring of kGroupStages buffers filled by asynchronous 16-byte copies (global -> shared, past
 // the registers), one tile ahead of the one being reduced, so every CTA always has loads in flight; two stages
 // rather than three leave room for a third CTA per SM, which is worth more (measured).
-template <typename T, int L, int CB>
+// REGS: a lane's share of the row (at most 128 bytes) is held in registers for both passes; otherwise both passes loop
+// over shared memory.
+template <typename T, int L, int CB, bool REGS>
 __global__ void __launch_bounds__(kGroupThreads, 8)
 score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__ labels, int64_t rows, int C,
                         int64_t ignore_index, float* __restrict__ row_loss, StatusBlock* status, uint32_t* hist0,
@@ -414,9 +416,9 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
         }
         __syncwarp();
         float m = -1e30f, s = 0.f;
-        if constexpr (VEC && L >= 8) {
-            // A lane's share of a row is at most 128 bytes (rows of up to 1024 and 2048 bytes over 8 and 16 lanes:
-            // the launcher never gives this path longer ones): it is read from shared memory once, into registers,
+        if constexpr (VEC && REGS) {
+            // A lane's share of a row is at most 128 bytes (the launcher gives this path rows of up to 1024 and 2048
+            // bytes over 8 and 16 lanes, never longer ones): it is read from shared memory once, into registers,
             // and both passes run from there, fully unrolled.  Round i (chunks i L .. i L + L - 1) is skipped by the whole warp once it is past the row.
             constexpr int CBV = VEC ? CB : 16;
             constexpr int kMaxCh = 128 / CBV;
@@ -447,8 +449,9 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
             unpack2(a1, t2, t3);
             s = (t0 + t1) + (t2 + t3);
         } else if constexpr (VEC) {
-            // short rows (4 lanes per row): a few chunks per lane, plain loops (measured faster here than the
-            // unrolled register copy above, whose fixed cost these rows do not repay)
+            // plain loops over the lane's chunks (4 lanes per row: measured faster than the unrolled register copy
+            // above, whose fixed cost short rows do not repay; 8 lanes per row on rows of 1 to 1.75 KB: a lane's
+            // share no longer fits 128 bytes, and half the lanes of the 16-lane variant still win)
             using Word = typename ChunkWord<VEC ? CB : 16>::type;
             const Word* xv = reinterpret_cast<const Word*>(x);
             const int nch = cls == 0 ? nchunk : 0;
@@ -1017,20 +1020,26 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
                                                      status, hist0, stage_bytes);
             err = cudaGetLastError();
         };
-        auto by_chunk = [&](auto lanes_tag) {
+        auto by_chunk = [&](auto lanes_tag, auto regs_tag) {
             constexpr int LN = decltype(lanes_tag)::value;
-            if (cb == 16) go(score_group_rows_kernel<T, LN, 16>, LN);
-            else if (cb == 8) go(score_group_rows_kernel<T, LN, 8>, LN);
+            constexpr bool RG = decltype(regs_tag)::value;
+            if (cb == 16) go(score_group_rows_kernel<T, LN, 16, RG>, LN);
+            else if (cb == 8) go(score_group_rows_kernel<T, LN, 8, RG>, LN);
             else if (cb == 4 && sizeof(T) == 2) {
-                if constexpr (sizeof(T) == 2) go(score_group_rows_kernel<T, LN, 4>, LN);  // (4-byte chunks of fp32 are single elements)
-            } else go(score_group_rows_kernel<T, LN, 0>, LN);
+                if constexpr (sizeof(T) == 2) go(score_group_rows_kernel<T, LN, 4, RG>, LN);  // (4-byte chunks of fp32 are single elements)
+            } else go(score_group_rows_kernel<T, LN, 0, false>, LN);
         };
-        // rows per tile (128 / L) times bytes per row: at most 25 KB per stage (32 x 800, 16 x 1024, 8 x 2048), plus padding.
-        // As few lanes per row as the row length allows: the per-row work is shared by 32 / L rows of a warp (measured
-        // at 600 and 800 bytes: 4 lanes 0.74-0.98 of the copy rate against 0.61-0.96 with 8; at 1000 bytes 8 lanes win)
-        if (row_bytes <= 800) by_chunk(std::integral_constant<int, 4>{});
-        else if (row_bytes <= 1024) by_chunk(std::integral_constant<int, 8>{});
-        else by_chunk(std::integral_constant<int, 16>{});
+        // rows per tile (128 / L) times bytes per row: at most 32 KB per stage (32 x 800, 16 x 2048, 8 x 2048), plus padding.
+        // As few lanes per row as the row length allows: the per-row work is shared by the 32 / L rows of a warp.
+        // Measured in one run, fraction of the copy rate: 600 and 800 bytes, 4 lanes 0.74-0.98 against 0.61-0.96 with
+        // 8; 1000 bytes, 8 lanes (share in registers) 0.74 against 0.64 with 4 and 0.67 with 8 looping; 1280-1600
+        // bytes, 8 lanes looping 0.86-1.02 against 0.71-0.97 with 16; 2000 bytes, fp32 1.00 with 8 lanes looping against
+        // 0.94 with 16, bf16 (twice the elements per byte) 0.71 against 0.79.
+        const bool vec = cb >= 8 || (cb == 4 && sizeof(T) == 2);
+        if (row_bytes <= 800) by_chunk(std::integral_constant<int, 4>{}, std::false_type{});
+        else if (row_bytes <= 1024) by_chunk(std::integral_constant<int, 8>{}, std::true_type{});
+        else if (row_bytes <= (sizeof(T) == 4 ? 2048 : 1792) && vec) by_chunk(std::integral_constant<int, 8>{}, std::false_type{});
+        else by_chunk(std::integral_constant<int, 16>{}, std::true_type{});
         return err;
     }
     if (row_bytes <= kStreamMaxRowBytes) {
