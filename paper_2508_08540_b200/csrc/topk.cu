@@ -206,6 +206,42 @@ __device__ void find_bin(const uint32_t* hist, int nbins, uint32_t& want, uint32
     __syncthreads();
 }
 
+// The same with two block barriers instead of five: every warp scans the warps' totals for itself.  `warp_tot` and
+// `result` must not be written again before another block barrier has been passed (none is taken at the end).
+template <bool GLOBAL>
+__device__ __forceinline__ void find_bin_fast(const uint32_t* hist, int nbins, uint32_t& want, uint32_t& bin, uint32_t* warp_tot, uint32_t* result) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool two = nbins == 2 * kThreads;
+    const int b0 = two ? nbins - 1 - 2 * static_cast<int>(threadIdx.x) : nbins - 1 - static_cast<int>(threadIdx.x);
+    const uint32_t c0 = GLOBAL ? __ldcg(hist + b0) : hist[b0];
+    const uint32_t c1 = !two ? 0u : GLOBAL ? __ldcg(hist + b0 - 1) : hist[b0 - 1];
+    const uint32_t c = c0 + c1;
+    uint32_t inc = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    const uint32_t wt = warp_tot[lane];
+    uint32_t winc = wt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, winc, o);
+        if (lane >= o) winc += n;
+    }
+    const uint32_t before = __shfl_sync(0xFFFFFFFFu, winc - wt, warp) + inc - c;
+    if (before < want && want <= before + c) {
+        const bool first = want <= before + c0;
+        result[0] = first ? b0 : b0 - 1;
+        result[1] = first ? want - before : want - before - c0;
+    }
+    __syncthreads();
+    bin = result[0];
+    want = result[1];
+}
+
 // Loads the E keys a thread owns (consecutive indices from `base`), 0 beyond N.  Key 0 belongs to no loss
 // (loss_key never returns it) and is below every threshold.
 template <int E>
@@ -569,26 +605,65 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
 }
 
 // ---------------------------------------------------------------------------
-// Pools of up to 65,536 entries: the same algorithm as ONE thread-block cluster, everything that blocks exchange
-// kept in (distributed) shared memory.  Block b owns a slice of 4,096 or 8,192 consecutive entries of the pool (in
-// registers) and sort tile b.  Digit histograms are added into block 0's shared memory and read from
-// there by every block; per-block counts, the sort's digit counts and the (key, index) pairs themselves are
-// written straight into the destination block's shared memory.  The barrier is the cluster's hardware barrier.
+// Pools of up to 65,536 entries: ONE thread-block cluster, everything that blocks exchange kept in (distributed)
+// shared memory.  Block b owns a slice of 4,096 or 8,192 consecutive entries of the pool (in registers).  Digit
+// histograms of the selection are added into block 0's shared memory; block 0 resolves the digit and tells every
+// block.  The barrier is the cluster's hardware barrier.  Two kernels:
+//   topk_cluster_kernel         index-ascending output: exact threshold (three digits), per-block counts, ordered
+//                               compaction straight into the output;
+//   topk_cluster_sorted_kernel  loss-descending output: see there.
 // ---------------------------------------------------------------------------
 namespace cg = cooperative_groups;
+
+// A 16-byte read from a shared-memory address of another block of the cluster (explicit instructions: reads written
+// one after the other are issued one after the other, before the first use).
+__device__ __forceinline__ uint4 ld_cluster_v4(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared::cluster.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
+// Digits `first`..`last` (0 = most significant) of the radix selection among the keys a cluster holds in registers.
+// hist_s: kSelBins zeroed words of this block (left zeroed); ghist: the workspace's [kSelPasses][kSelBins] histograms,
+// those of the digits asked for zeroed.  Every block adds its counts to the global histogram, and after ONE cluster
+// barrier every block resolves the digit for itself.  (Adding them into block 0's shared memory instead cost 1.2 to 2.4 us
+// a digit for the additions alone, all aimed at one multiprocessor, plus a second barrier to spread the answer.)
+// On return `prefix` holds the resolved digits and `want` the rank left inside that prefix.
+template <int CE>
+__device__ __forceinline__ void cluster_select_digits(cg::cluster_group& cluster, const uint32_t (&key)[CE], int first, int last,
+                                                      uint32_t* hist_s, uint32_t* ghist, uint32_t* warp_tot, uint32_t* result,
+                                                      uint32_t& prefix, uint32_t& want) {
+    const int tid = threadIdx.x;
+    for (int pass = first; pass <= last; ++pass) {
+        const uint32_t mask = prefix_mask(pass);
+        __syncthreads();  // hist_s is zero
+#pragma unroll
+        for (int i = 0; i < CE; ++i) {
+            const bool in = key[i] != 0u && (key[i] & mask) == prefix;
+            // plain shared-memory atomics: measured faster than warp-aggregated ones (match.any) for crowded, uniform and
+            // all-equal keys alike
+            if (in) atomicAdd(&hist_s[digit_of(key[i], pass)], 1u);
+        }
+        __syncthreads();
+        for (int i = tid; i < kSelBins; i += kThreads) {
+            const uint32_t c = hist_s[i];
+            if (c) atomicAdd(ghist + pass * kSelBins + i, c);
+            hist_s[i] = 0;
+        }
+        cluster.sync();  // every block's additions are in
+        uint32_t bin;
+        find_bin_fast<true>(ghist + pass * kSelBins, pass == 2 ? 1024 : kSelBins, want, bin, warp_tot, result);
+        prefix |= pass == 0 ? bin << 21 : pass == 1 ? bin << 10 : bin;
+    }
+}
 
 // CE keys per thread (blocks of 1024 CE entries), at most CB blocks: 4 x 16 (a cluster of more than 8 blocks needs the
 // device's consent, see launch_topk) or 8 x 8.
 template <int CE, int CB>
 struct ClusterLayout {
     static constexpr int kTile = kThreads * CE;
-    static constexpr size_t kCountersBytes = sizeof(uint32_t) * kWarps * kCounterPitch;
-    static constexpr size_t kPairsBytes = sizeof(uint2) * 2 * kTile;
-    static constexpr size_t kMatBytes = sizeof(uint32_t) * CB * kSortBins;
-    static constexpr size_t kSmemBytes = kCountersBytes + kPairsBytes + kMatBytes + sizeof(uint4) * CB;
-    static_assert(kCountersBytes % 16 == 0, "the pair buffers start 16-byte aligned");
-    static_assert(sizeof(uint32_t) * kSelPasses * kSelBins <= kPairsBytes / 2, "the selection's histograms fit in the first pair buffer");
-    static_assert(kTile <= 1024 * kSortMaxRounds, "a block's pairs are one sort tile");
+    static constexpr size_t kHistBytes = sizeof(uint32_t) * kSelBins;
+    static constexpr size_t kSmemBytes = kHistBytes + sizeof(uint4) * CB;
 };
 
 template <int CE, int CB>
@@ -596,242 +671,425 @@ __global__ void __launch_bounds__(kThreads, 1) topk_cluster_kernel(const __grid_
     using Lay = ClusterLayout<CE, CB>;
     constexpr int kClE = CE, kClTile = Lay::kTile;
     extern __shared__ __align__(16) unsigned char cl_smem[];
-    uint32_t* dyn = reinterpret_cast<uint32_t*>(cl_smem);                                          // hist_s, later counters
-    uint2* pairs = reinterpret_cast<uint2*>(cl_smem + Lay::kCountersBytes);                         // [2][kClTile]
-    uint32_t* acc_hist = reinterpret_cast<uint32_t*>(pairs);                                        // block 0, selection only: [3][kSelBins]
-    uint32_t* mat = reinterpret_cast<uint32_t*>(cl_smem + Lay::kCountersBytes + Lay::kPairsBytes);   // [blocks][kSortBins]
-    uint4* cta_cnt = reinterpret_cast<uint4*>(cl_smem + Lay::kCountersBytes + Lay::kPairsBytes + Lay::kMatBytes);
+    uint32_t* hist_s = reinterpret_cast<uint32_t*>(cl_smem);
+    uint4* cta_cnt = reinterpret_cast<uint4*>(cl_smem + Lay::kHistBytes);
     __shared__ uint32_t warp_tot[kWarps + 1];
     __shared__ uint32_t result[2];
-    __shared__ uint32_t red[3];
-    __shared__ uint32_t digit_s[2];  // (bin, rank left) of the digit block 0 resolved last
-    __shared__ uint32_t base_s[kSortBins], tot_s[kSortBins], half_cnt[2][kSortBins];
+    __shared__ uint32_t red[2];
+    cg::cluster_group cluster = cg::this_cluster();
+    const int tid = threadIdx.x, lane = tid & 31;
+    const uint32_t rank = blockIdx.x, nblocks = gridDim.x;
+    const float* __restrict__ losses = p.losses;
+    const int64_t N = p.N;
+
+    for (int i = tid; i < kSelBins; i += kThreads) hist_s[i] = 0;
+    if (tid < 2) red[tid] = 0;
+    grid_dependency_wait();  // the losses (and the scorer's histogram) are complete from here on
+
+    if (p.standalone) {
+        // a selection on its own: the status block reads "nothing to report", and block 0 clears the workspace's
+        // histograms (a fused call's memset has done both)
+        if (rank == 0) {
+            if (tid == 0) {
+                p.ws.status->bad_labels = 0;
+                p.ws.status->timeout = 0;
+            }
+            for (int i = tid; i < kSelPasses * kSelBins; i += kThreads) p.ws.hist[i] = 0;
+        }
+        cluster.sync();
+    }
+    uint32_t key[kClE];
+    load_keys<kClE>(losses, N, static_cast<int64_t>(rank) * kClTile + static_cast<int64_t>(tid) * kClE, key);
+
+    // ---- 1. radix select: the key T of the k-th entry and r, the entries equal to T that are still selected ----
+    uint32_t prefix = 0, want = p.k;
+    if (p.hist0_ready) {
+        uint32_t bin;
+        find_bin_fast<true>(p.ws.hist, kSelBins, want, bin, warp_tot, result);
+        prefix = bin << 21;
+    }
+    cluster_select_digits<kClE>(cluster, key, p.hist0_ready ? 1 : 0, kSelPasses - 1, hist_s, p.ws.hist, warp_tot, result, prefix, want);
+    const uint32_t T = prefix, r = want;
+
+    // ---- 2. per block: keys above T, keys equal to T; every block gets every block's ----
+    uint32_t my_gt = 0, my_eq = 0;
+    {
+#pragma unroll
+        for (int i = 0; i < kClE; ++i) {
+            my_gt += key[i] > T;
+            my_eq += key[i] == T;
+        }
+        uint32_t packed = my_gt | (my_eq << 16);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) packed += __shfl_xor_sync(0xFFFFFFFFu, packed, o);
+        if (lane == 0) {
+            atomicAdd(&red[0], packed & 0xFFFFu);
+            atomicAdd(&red[1], packed >> 16);
+        }
+        __syncthreads();
+        if (tid < static_cast<int>(nblocks)) cluster.map_shared_rank(cta_cnt, tid)[rank] = make_uint4(red[0], red[1], 0u, 0u);
+    }
+    cluster.sync();  // the last access to another block's shared memory is before this barrier
+
+    // ---- 3. ordered compaction, straight into the output ----
+    uint32_t gt_before = 0, eq_before = 0;
+    for (uint32_t b = 0; b < rank; ++b) {
+        const uint4 c = cta_cnt[b];
+        gt_before += c.x;
+        eq_before += c.y;
+    }
+    const uint32_t packed = block_exclusive_scan(my_gt | (my_eq << 16), warp_tot);
+    uint32_t gt_run = gt_before + (packed & 0xFFFFu);
+    uint32_t eq_run = eq_before + (packed >> 16);
+    const int64_t base = static_cast<int64_t>(rank) * kClTile + static_cast<int64_t>(tid) * kClE;
+#pragma unroll
+    for (int i = 0; i < kClE; ++i) {
+        const bool above = key[i] > T;
+        const bool tie = key[i] == T;
+        if (above || (tie && eq_run < r)) {
+            const uint32_t pos = gt_run + min(eq_run, r);
+            const int64_t j = base + i;
+            p.out_idx[pos] = static_cast<int32_t>(j);
+            if (p.out_vals) p.out_vals[pos] = losses[j];
+        }
+        gt_run += above;
+        eq_run += tie;
+    }
+}
+
+// Loss-descending output.  The selection stops after two digits: every key that shares the 22 resolved bits with the
+// k-th key, or lies above them, is a candidate (k' >= k of them: k plus the few keys in the k-th key's bin of 1,024
+// consecutive keys).  The candidates are sorted whole, stably, by v = key - T (T = the lowest key of that bin) in
+// descending 9-bit digits, least significant first; the first k positions of the result are the selection, ties
+// between equal keys in index order because the candidates start in index order.  No threshold has to be exact and
+// no tie has to be counted before the sort.
+//
+// One cluster barrier per sort pass.  The digit histograms of ALL passes are taken at once from the registers, so
+// where a digit's run starts is known up front; what a pass still needs, how many entries with the same digit sit in
+// the tiles before a block's own, is counted one pass ahead: while a block scatters its entries it counts, per
+// destination tile, the NEXT digit of what it sends there (flow[t][d]), turns the counts into running sums over t,
+// and after the barrier the owner of tile t adds up row t of every block's matrix.  Reading another block's shared
+// memory is slow (some 30 KB per microsecond and block, measured), so these counts travel as 16-bit halves (no
+// block holds more than 8,192 entries) and every read is issued together with seven others.
+// Sort tile b (1,024 R consecutive positions, R = 1, 2, 4 or 8 as k' needs) is block b's pair buffer.  For pass 0 every
+// warp first packs the candidates among its 32 CE entries (dealt to its lanes so that rounds run through consecutive
+// indices), in order, into a list of its own, which it then treats like a slice of a tile.
+template <int CE, int CB>
+struct SortedClusterLayout {
+    static constexpr int kTile = kThreads * CE;
+    static constexpr size_t kCountersBytes = sizeof(uint16_t) * kWarps * kSortBins;  // per-warp digit counters; the selection's hist_s before
+    static constexpr size_t kPairsBytes = sizeof(uint2) * 2 * kTile;                 // two (key, index) buffers
+    static constexpr size_t kFlowBytes = sizeof(uint16_t) * 2 * CB * kSortBins;      // flow[2][CB][kSortBins]; the second one holds the four digit histograms first
+    static constexpr size_t kSmemBytes = kCountersBytes + kPairsBytes + kFlowBytes;
+    static_assert(sizeof(uint32_t) * kSelBins <= kCountersBytes, "the selection's block histogram fits in the counters");
+    static_assert(4 <= CB, "the digit histograms fit in one flow matrix");
+    static_assert(CE <= kSortMaxRounds && kTile <= 8192 && kTile < 65536, "a block's digit counts fit 16 bits");
+};
+
+template <int CE, int CB>
+__global__ void __launch_bounds__(kThreads, 1) topk_cluster_sorted_kernel(const __grid_constant__ SelectParams p) {
+    using Lay = SortedClusterLayout<CE, CB>;
+    constexpr int kClTile = Lay::kTile;
+    constexpr int kRowWords = kSortBins / 2;      // one row of 16-bit digit counts, in 32-bit words
+    constexpr int kFlowWords = CB * kRowWords;
+    constexpr int kDigits = 4;  // 9 + 9 + 9 + 5 bits
+    extern __shared__ __align__(16) unsigned char cl_smem[];
+    uint32_t* hist_s = reinterpret_cast<uint32_t*>(cl_smem);
+    uint16_t(*counters)[kSortBins] = reinterpret_cast<uint16_t(*)[kSortBins]>(cl_smem);
+    uint2* pairs = reinterpret_cast<uint2*>(cl_smem + Lay::kCountersBytes);
+    uint32_t* flow = reinterpret_cast<uint32_t*>(cl_smem + Lay::kCountersBytes + Lay::kPairsBytes);  // [2][CB][kRowWords], two digits a word
+    uint32_t* dig_hist = flow + kFlowWords;                                                          // [kDigits][kRowWords]
+    __shared__ uint32_t warp_tot[kWarps + 1];
+    __shared__ uint32_t result[2];
+    __shared__ uint32_t vmax_s, vmax_all_s;
+    __shared__ uint32_t warp_sum[kWarps];
+    __shared__ uint32_t acc_s[2][kRowWords];  // sums of what is read from the other blocks, two digits a word: all of them; the blocks before this one
+    __shared__ __align__(16) uint32_t base_s[kDigits][kSortBins];  // entries whose digit is larger, per pass
+    __shared__ __align__(16) uint32_t tilebase_s[kSortBins];       // the same plus the entries of the same digit in the tiles before this one
+    __shared__ uint32_t half_cnt[2][kSortBins];
     cg::cluster_group cluster = cg::this_cluster();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t rank = blockIdx.x, nblocks = gridDim.x;
     const float* __restrict__ losses = p.losses;
     const int64_t N = p.N;
-    uint32_t* hist_s = dyn;
+    const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
 
     for (int i = tid; i < kSelBins; i += kThreads) hist_s[i] = 0;
-    for (int i = tid; i < kSelPasses * kSelBins; i += kThreads) acc_hist[i] = 0;
-    for (int i = tid; i < CB * kSortBins; i += kThreads) mat[i] = 0;
-    if (tid < 3) red[tid] = 0;
-    cluster.sync();          // every block's accumulators are clear before anybody adds to them
+    for (int i = tid; i < 2 * kFlowWords / 4; i += kThreads) reinterpret_cast<uint4*>(flow)[i] = zero4;
+    if (tid < 2 * kRowWords) acc_s[0][tid] = 0;
+    if (tid == 0) vmax_s = 0;
     grid_dependency_wait();  // the losses (and the scorer's histogram) are complete from here on
 
-    if (p.standalone && rank == 0 && tid == 0) {  // a selection on its own: the status block reads "nothing to report"
-        p.ws.status->bad_labels = 0;
-        p.ws.status->timeout = 0;
+    // The cluster's digit totals of sort passes 1 to 3 are added up in global memory too, in the workspace's third
+    // selection histogram (this kernel resolves two digits only).
+    uint32_t* digit_totals = p.ws.hist + 2 * kSelBins;  // [3][kSortBins]
+    if (p.standalone) {
+        // a selection on its own: the status block reads "nothing to report", and block 0 clears the workspace's
+        // histograms (a fused call's memset has done both)
+        if (rank == 0) {
+            if (tid == 0) {
+                p.ws.status->bad_labels = 0;
+                p.ws.status->timeout = 0;
+            }
+            for (int i = tid; i < kSelPasses * kSelBins; i += kThreads) p.ws.hist[i] = 0;
+        }
+        cluster.sync();
     }
-    uint32_t key[kClE];
-    load_keys<kClE>(losses, N, static_cast<int64_t>(rank) * kClTile + static_cast<int64_t>(tid) * kClE, key);
+    // entry (round i, lane l) of warp w: index block start + 32 CE w + 32 i + l
+    const int64_t wbase = static_cast<int64_t>(rank) * kClTile + static_cast<int64_t>(warp) * (32 * CE) + lane;
+    uint32_t key[CE];
+#pragma unroll
+    for (int i = 0; i < CE; ++i) {
+        const int64_t j = wbase + 32 * i;
+        key[i] = j < N ? loss_key(losses[j]) : 0u;
+    }
 
-    // ---- 1. radix select ----
+    // ---- 1. the two leading digits of the k-th key ----
     uint32_t prefix = 0, want = p.k;
     if (p.hist0_ready) {
         uint32_t bin;
-        find_bin(p.ws.hist, kSelBins, want, bin, warp_tot, result);
+        find_bin_fast<true>(p.ws.hist, kSelBins, want, bin, warp_tot, result);
         prefix = bin << 21;
     }
-    for (int pass = p.hist0_ready ? 1 : 0; pass < kSelPasses; ++pass) {
-        const uint32_t mask = prefix_mask(pass);
-        __syncthreads();  // hist_s is zero
-#pragma unroll
-        for (int i = 0; i < kClE; ++i) {
-            const bool in = key[i] != 0u && (key[i] & mask) == prefix;
-            // plain shared-memory atomics: measured faster than warp-aggregated ones (match.any) for crowded, uniform and
-            // all-equal keys alike
-            if (in) atomicAdd(&hist_s[digit_of(key[i], pass)], 1u);
-        }
-        __syncthreads();
-        uint32_t* acc0 = cluster.map_shared_rank(acc_hist, 0) + pass * kSelBins;
-        for (int i = tid; i < kSelBins; i += kThreads) {
-            const uint32_t c = hist_s[i];
-            if (c) atomicAdd(acc0 + i, c);
-            hist_s[i] = 0;
-        }
-        cluster.sync();
-        // block 0 resolves the digit from its own shared memory and tells every block (reading 2,048 bins of
-        // another block's shared memory from every block took longer than this second barrier)
-        if (rank == 0) {
-            uint32_t bin;
-            find_bin<false>(acc_hist + pass * kSelBins, pass == 2 ? 1024 : kSelBins, want, bin, warp_tot, result);
-            if (tid < static_cast<int>(nblocks)) {
-                uint32_t* dst = cluster.map_shared_rank(digit_s, tid);
-                dst[0] = bin;
-                dst[1] = want;
-            }
-        }
-        cluster.sync();
-        const uint32_t bin = digit_s[0];
-        want = digit_s[1];
-        prefix |= pass == 0 ? bin << 21 : pass == 1 ? bin << 10 : bin;
-    }
-    const uint32_t T = prefix, r = want;
+    cluster_select_digits<CE>(cluster, key, p.hist0_ready ? 1 : 0, 1, hist_s, p.ws.hist, warp_tot, result, prefix, want);
+    const uint32_t T = prefix;  // candidates: key >= T (and a real key: padding is 0)
 
-    // ---- 2. per block: keys above T, keys equal to T, largest key; every block gets every block's ----
-    uint32_t my_gt = 0, my_eq = 0;
+    // ---- 2. this block's digit histograms of v = key - T for all passes, its largest v, and each warp's
+    //         candidates packed in index order into the second pair buffer ----
+    uint2* stage = pairs + kClTile + warp * (32 * CE);
+    uint32_t cnt_w = 0;  // entries this warp ranks in the coming pass
     {
-        uint32_t mx = 0;
+        uint32_t vm = 0;
 #pragma unroll
-        for (int i = 0; i < kClE; ++i) {
-            my_gt += key[i] > T;
-            my_eq += key[i] == T;
-            mx = max(mx, key[i]);
+        for (int i = 0; i < CE; ++i) {
+            const bool cand = key[i] != 0u && key[i] >= T;
+            const uint32_t votes = __ballot_sync(0xFFFFFFFFu, cand);
+            if (cand) {
+                const uint32_t v = key[i] - T;
+                vm = max(vm, v);
+                const uint32_t d0 = v & (kSortBins - 1), d1 = (v >> kSortBits) & (kSortBins - 1), d2 = (v >> (2 * kSortBits)) & (kSortBins - 1),
+                               d3 = v >> (3 * kSortBits);
+                atomicAdd(&dig_hist[d0 >> 1], 1u << ((d0 & 1u) * 16));
+                atomicAdd(&dig_hist[kRowWords + (d1 >> 1)], 1u << ((d1 & 1u) * 16));
+                atomicAdd(&dig_hist[2 * kRowWords + (d2 >> 1)], 1u << ((d2 & 1u) * 16));
+                atomicAdd(&dig_hist[3 * kRowWords + (d3 >> 1)], 1u << ((d3 & 1u) * 16));
+                stage[cnt_w + __popc(votes & ((1u << lane) - 1u))] = make_uint2(key[i], static_cast<uint32_t>(wbase + 32 * i));
+            }
+            cnt_w += __popc(votes);
         }
-        uint32_t packed = my_gt | (my_eq << 16);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            packed += __shfl_xor_sync(0xFFFFFFFFu, packed, o);
-            mx = max(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-        }
-        if (lane == 0) {
-            atomicAdd(&red[0], packed & 0xFFFFu);
-            atomicAdd(&red[1], packed >> 16);
-            atomicMax(&red[2], mx);
-        }
-        __syncthreads();
-        if (tid < static_cast<int>(nblocks)) cluster.map_shared_rank(cta_cnt, tid)[rank] = make_uint4(red[0], red[1], red[2], 0u);
+        for (int o = 16; o > 0; o >>= 1) vm = max(vm, __shfl_xor_sync(0xFFFFFFFFu, vm, o));
+        if (lane == 0 && vm) atomicMax(&vmax_s, vm);
+    }
+    __syncthreads();
+    if (tid < 3 * kRowWords) {  // passes 1 to 3: this block's counts into the cluster's totals
+        const uint32_t w = dig_hist[kRowWords + tid];
+        if (w & 0xFFFFu) atomicAdd(&digit_totals[2 * tid], w & 0xFFFFu);
+        if (w >> 16) atomicAdd(&digit_totals[2 * tid + 1], w >> 16);
     }
     cluster.sync();
 
-    // ---- 3. ordered compaction ----
-    uint32_t gt_before = 0, eq_before = 0, kmax = 0;
-    for (uint32_t b = 0; b < nblocks; ++b) {
-        const uint4 c = cta_cnt[b];
-        gt_before += b < rank ? c.x : 0u;
-        eq_before += b < rank ? c.y : 0u;
-        kmax = max(kmax, c.z);
-    }
-    const uint32_t range = kmax - T;
-    const int passes = p.order == LSGD_ORDER_INDEX_ASC ? 0 : (32 - __clz(range) + kSortBits - 1) / kSortBits;
-    const bool direct = passes == 0;
-    const int R = p.sort_rounds;
-    const int tshift = 10 + (R == 1 ? 0 : R == 2 ? 1 : R == 4 ? 2 : 3);
-    const uint32_t tmask = (1u << tshift) - 1u;
-    const uint32_t St = p.sort_tiles;  // <= nblocks: sort tile b lives in block b
+    // ---- 3. all blocks' histograms: where each digit's run starts in every pass (larger digits first), the number
+    //         of candidates, the number of passes ----
+    uint32_t kc;  // k', the candidates
     {
-        const uint32_t packed = block_exclusive_scan(my_gt | (my_eq << 16), warp_tot);
-        uint32_t gt_run = gt_before + (packed & 0xFFFFu);
-        uint32_t eq_run = eq_before + (packed >> 16);
-        const int64_t base = static_cast<int64_t>(rank) * kClTile + static_cast<int64_t>(tid) * kClE;
+        // Pass 0 needs every block's histogram (how many candidates with the same digit sit in the blocks before this
+        // one): thread (other block u, 16-byte piece) reads one piece and adds it to this block's sums, two digits a word
+        // (the other blocks hold fewer than 65,536 entries together: no half carries).  Block u is counted from this
+        // block's successor, so that no block is read by all at once.  The totals of the later passes come from global memory.
+        const uint32_t g1 = __ldcg(digit_totals + tid), g2 = tid < kSortBins ? __ldcg(digit_totals + kThreads + tid) : 0u;
+        {
+            const int u = tid >> 6, piece = tid & 63;
+            if (u < static_cast<int>(nblocks) - 1) {
+                uint32_t b = rank + 1 + u;
+                b -= b >= nblocks ? nblocks : 0u;
+                uint32_t ra;
+                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(static_cast<uint32_t>(__cvta_generic_to_shared(dig_hist + 4 * piece))), "r"(b));
+                const uint4 c = ld_cluster_v4(ra);
+                const uint32_t w[4] = {c.x, c.y, c.z, c.w};
 #pragma unroll
-        for (int i = 0; i < kClE; ++i) {
-            const bool above = key[i] > T;
-            const bool tie = key[i] == T;
-            if (above || (tie && eq_run < r)) {
-                const uint32_t pos = gt_run + min(eq_run, r);
-                const int64_t j = base + i;
-                if (direct) {
-                    p.out_idx[pos] = static_cast<int32_t>(j);
-                    if (p.out_vals) p.out_vals[pos] = losses[j];
-                } else {
-                    cluster.map_shared_rank(pairs, pos >> tshift)[pos & tmask] = make_uint2(key[i], static_cast<uint32_t>(j));
+                for (int e = 0; e < 4; ++e) {
+                    if (w[e]) {
+                        atomicAdd(&acc_s[0][4 * piece + e], w[e]);
+                        if (b < rank) atomicAdd(&acc_s[1][4 * piece + e], w[e]);
+                    }
                 }
             }
-            gt_run += above;
-            eq_run += tie;
         }
+        if (warp == kWarps - 1) {  // (never one of the readers above)
+            uint32_t m = lane < static_cast<int>(nblocks) ? *cluster.map_shared_rank(&vmax_s, lane) : 0u;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+            if (lane == 0) vmax_all_s = m;
+        }
+        base_s[1 + (tid >> 9)][tid & (kSortBins - 1)] = g1;
+        if (tid < kSortBins) base_s[3][tid] = g2;
+        for (int i = tid; i < static_cast<int>(Lay::kCountersBytes / 16); i += kThreads) reinterpret_cast<uint4*>(cl_smem)[i] = zero4;
+        __syncthreads();
+        // thread (pass q, pair j): digits 511 - 2 j and 510 - 2 j; a descending exclusive scan per pass
+        const int q = tid >> 8, j = tid & 255, lo = kSortBins - 2 - 2 * j;
+        uint32_t g_lo, g_hi, b_lo = 0, b_hi = 0;
+        if (q == 0) {
+            const uint32_t wo = acc_s[0][lo / 2], wb = acc_s[1][lo / 2], wm = dig_hist[lo / 2];
+            acc_s[0][lo / 2] = 0;  // clear again for the next pass's sums
+            acc_s[1][lo / 2] = 0;
+            g_lo = (wo & 0xFFFFu) + (wm & 0xFFFFu), g_hi = (wo >> 16) + (wm >> 16);
+            b_lo = wb & 0xFFFFu, b_hi = wb >> 16;
+        } else {
+            g_lo = base_s[q][lo], g_hi = base_s[q][lo + 1];
+        }
+        const uint32_t s2 = g_lo + g_hi;
+        uint32_t inc = s2;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= o) inc += n;
+        }
+        if (lane == 31) warp_sum[warp] = inc;
+        __syncthreads();
+        uint32_t below = 0;  // entries of this pass with larger digits, in the warps before this one
+#pragma unroll
+        for (int w = 0; w < 8; ++w) below += w < (warp & 7) ? warp_sum[(warp & ~7) + w] : 0u;
+        const uint32_t start_hi = below + inc - s2;
+        base_s[q][lo + 1] = start_hi;
+        base_s[q][lo] = start_hi + g_hi;
+        if (q == 0) {
+            tilebase_s[lo + 1] = start_hi + b_hi;
+            tilebase_s[lo] = start_hi + g_hi + b_lo;
+        }
+        kc = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) kc += warp_sum[w];
     }
-    if (direct) return;  // nobody touches another block's shared memory after the barrier above
-    cluster.sync();
-
-    // ---- 4. stable LSD sort on u = kmax - key, 9 bits per pass; tile b = block b's pair buffer ----
-    uint32_t(*counters)[kCounterPitch] = reinterpret_cast<uint32_t(*)[kCounterPitch]>(dyn);
+    const uint32_t vmax = vmax_all_s;
+    const int passes = max(1, (32 - __clz(vmax) + kSortBits - 1) / kSortBits);
+    int R = 1;
+    while (nblocks * 1024u * R < kc) R <<= 1;  // R <= CE: the candidates are no more than the pool
+    const int tshift = 10 + (R == 1 ? 0 : R == 2 ? 1 : R == 4 ? 2 : 3);
+    const uint32_t tmask = (1u << tshift) - 1u;
     const uint32_t k = p.k;
-    const bool has_tile = rank < St;
-    const uint32_t first = (rank << tshift) + warp * (R * 32);  // global position of this warp's first entry
+
+    // ---- 4. the passes: pass 0 from the warps' packed lists, the others tile b in block b ----
+    const uint32_t first = (rank << tshift) + warp * (R * 32);  // position of this warp's first entry in passes 1, 2, ...
+    uint32_t* cnt32 = reinterpret_cast<uint32_t*>(cl_smem);     // the counters, two digits a word
     for (int pass = 0; pass < passes; ++pass) {
         const bool last = pass == passes - 1;
         const int shift = kSortBits * pass;
-        const uint2* pairs_in = pairs + (pass & 1) * kClTile;
-        uint2* pairs_out = pairs + ((pass + 1) & 1) * kClTile;
+        uint2* pairs_out = pairs + (pass & 1) * kClTile;
+        uint32_t* flow_out = flow + (pass & 1) * kFlowWords;
+        const uint2* src = stage;
+        if (pass > 0) {
+            const uint32_t* flow_in = flow + ((pass - 1) & 1) * kFlowWords;
+            {
+                // row `rank` of every block's matrix: thread (block u, 16-byte piece) reads one piece and adds it to this
+                // block's sums (what is summed lies in the tiles before this block's own: fewer than 65,536 entries
+                // whenever this tile holds any, so no half carries)
+                const int u = tid >> 6, piece = tid & 63;
+                if (u < static_cast<int>(nblocks)) {
+                    uint32_t b = rank + u;
+                    b -= b >= nblocks ? nblocks : 0u;
+                    uint32_t ra;
+                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(static_cast<uint32_t>(__cvta_generic_to_shared(flow_in + rank * kRowWords + 4 * piece))), "r"(b));
+                    const uint4 c = ld_cluster_v4(ra);
+                    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (w[e]) atomicAdd(&acc_s[0][4 * piece + e], w[e]);
+                }
+            }
+            for (int i = tid; i < static_cast<int>(Lay::kCountersBytes / 16); i += kThreads) reinterpret_cast<uint4*>(cl_smem)[i] = zero4;
+            if (!last)
+                for (int i = tid; i < kFlowWords / 4; i += kThreads) reinterpret_cast<uint4*>(flow_out)[i] = zero4;
+            src = pairs + ((pass - 1) & 1) * kClTile + warp * (R * 32);
+            cnt_w = first < kc ? min(kc - first, static_cast<uint32_t>(R * 32)) : 0u;
+        }
+        // after its last read of another block's shared memory a block signals the barrier that it waits for before it exits
+        if (last) cluster.barrier_arrive();
         uint32_t skey[kSortMaxRounds], srank[kSortMaxRounds];
         int32_t sidx[kSortMaxRounds];
-        if (has_tile) {
-            for (int i = tid; i < kWarps * kCounterPitch; i += kThreads) dyn[i] = 0;
 #pragma unroll
-            for (int rd = 0; rd < kSortMaxRounds; ++rd) {
-                const uint32_t e = first + rd * 32 + lane;
-                const bool live = rd < R && e < k;
-                const uint2 pr = live ? pairs_in[e & tmask] : make_uint2(0u, 0u);
-                skey[rd] = pr.x;
-                sidx[rd] = static_cast<int32_t>(pr.y);
+        for (int rd = 0; rd < kSortMaxRounds; ++rd) {
+            const uint32_t e = rd * 32 + lane;
+            const uint2 pr = e < cnt_w ? src[e] : make_uint2(T, 0u);
+            skey[rd] = pr.x;
+            sidx[rd] = static_cast<int32_t>(pr.y);
+        }
+        __syncthreads();  // counters are zero (pass 0: and the bases are written)
+        if (pass > 0 && tid < kRowWords) {
+            const uint32_t w = acc_s[0][tid];
+            acc_s[0][tid] = 0;
+            tilebase_s[2 * tid] = base_s[pass][2 * tid] + (w & 0xFFFFu);
+            tilebase_s[2 * tid + 1] = base_s[pass][2 * tid + 1] + (w >> 16);
+        }
+        // rank by digit within the warp, in round-then-lane order; the warp's digit counts end up in its counter row
+#pragma unroll
+        for (int rd = 0; rd < kSortMaxRounds; ++rd) {
+            if (rd * 32 < cnt_w) {
+                const bool live = rd * 32 + lane < cnt_w;
+                const uint32_t dd = ((skey[rd] - T) >> shift) & (kSortBins - 1);
+                const uint32_t peers = match_digit(dd, live);
+                const int leader = live ? __ffs(peers) - 1 : lane;
+                uint32_t old = 0;
+                if (live && lane == leader) {
+                    old = counters[warp][dd];
+                    counters[warp][dd] = static_cast<uint16_t>(old + __popc(peers));
+                }
+                old = __shfl_sync(0xFFFFFFFFu, old, leader);
+                srank[rd] = old + __popc(peers & ((1u << lane) - 1u));
+                __syncwarp();
             }
-            __syncthreads();
+        }
+        __syncthreads();
+        if (tid < kSortBins) {  // per pair of digits, the exclusive prefix of the warps' counts within each half of the block
+            const int dp = tid & (kRowWords - 1), h = tid / kRowWords;
+            constexpr int kHalf = kWarps / 2;
+            uint32_t c[kHalf];
 #pragma unroll
-            for (int rd = 0; rd < kSortMaxRounds; ++rd) {
-                if (rd < R) {
-                    const uint32_t e = first + rd * 32 + lane;
-                    const bool live = e < k;
-                    const uint32_t dd = ((kmax - skey[rd]) >> shift) & (kSortBins - 1);
-                    const uint32_t peers = match_digit(dd, live);
-                    const int leader = live ? __ffs(peers) - 1 : lane;
-                    uint32_t old = 0;
-                    if (live && lane == leader) {
-                        old = counters[warp][dd];
-                        counters[warp][dd] = old + __popc(peers);
+            for (int u = 0; u < kHalf; ++u) c[u] = cnt32[(kHalf * h + u) * kRowWords + dp];
+            uint32_t run = 0;
+#pragma unroll
+            for (int u = 0; u < kHalf; ++u) {
+                cnt32[(kHalf * h + u) * kRowWords + dp] = run;
+                run += c[u];  // at most 16 x 256 a digit: the halves never carry
+            }
+            half_cnt[h][2 * dp] = run & 0xFFFFu;
+            half_cnt[h][2 * dp + 1] = run >> 16;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int rd = 0; rd < kSortMaxRounds; ++rd) {
+            if (rd * 32 + lane < cnt_w) {
+                const uint32_t v = skey[rd] - T, dd = (v >> shift) & (kSortBins - 1);
+                const uint32_t pos = tilebase_s[dd] + counters[warp][dd] + (warp >= kWarps / 2 ? half_cnt[0][dd] : 0u) + srank[rd];
+                if (last) {
+                    if (pos < k) {
+                        p.out_idx[pos] = sidx[rd];
+                        if (p.out_vals) p.out_vals[pos] = loss_of_key(skey[rd], losses, sidx[rd]);
                     }
-                    old = __shfl_sync(0xFFFFFFFFu, old, leader);
-                    srank[rd] = old + __popc(peers & ((1u << lane) - 1u));
-                    __syncwarp();
+                } else {
+                    const uint32_t t = pos >> tshift, dn = (v >> (shift + kSortBits)) & (kSortBins - 1);
+                    atomicAdd(&flow_out[t * kRowWords + (dn >> 1)], 1u << ((dn & 1u) * 16));
+                    cluster.map_shared_rank(pairs_out, t)[pos & tmask] = make_uint2(skey[rd], static_cast<uint32_t>(sidx[rd]));
                 }
             }
+        }
+        if (!last) {
             __syncthreads();
-            {   // per digit, exclusive prefix of the warps' counts within each half of the block: thread (digit, half)
-                const int d = tid & (kSortBins - 1), h = tid / kSortBins;
-                constexpr int kHalf = kWarps / 2;
-                uint32_t c[kHalf];
+            if (tid < kRowWords) {  // counts per destination tile -> running sums over the tiles (two digits a word, no carries)
+                uint32_t c[CB];
 #pragma unroll
-                for (int u = 0; u < kHalf; ++u) c[u] = counters[kHalf * h + u][d];
+                for (int t = 0; t < CB; ++t) c[t] = t < static_cast<int>(nblocks) ? flow_out[t * kRowWords + tid] : 0u;
                 uint32_t run = 0;
 #pragma unroll
-                for (int u = 0; u < kHalf; ++u) {
-                    counters[kHalf * h + u][d] = run;
-                    run += c[u];
+                for (int t = 0; t < CB; ++t) {
+                    if (t < static_cast<int>(nblocks)) flow_out[t * kRowWords + tid] = run;
+                    run += c[t];
                 }
-                half_cnt[h][d] = run;
             }
-            __syncthreads();
-            // this tile's digit counts, into every block's copy of the count matrix
-            for (uint32_t i = tid; i < nblocks * kSortBins; i += kThreads) {
-                const uint32_t b = i / kSortBins, d = i % kSortBins;
-                cluster.map_shared_rank(mat, b)[rank * kSortBins + d] = half_cnt[0][d] + half_cnt[1][d];
-            }
+            cluster.sync();
         }
-        cluster.sync();
-        if (has_tile) {
-            {
-                uint32_t total = 0, before = 0;
-                if (tid < kSortBins) {
-                    for (uint32_t b = 0; b < St; ++b) {
-                        const uint32_t c = mat[b * kSortBins + tid];
-                        total += c;
-                        before += b < rank ? c : 0u;
-                    }
-                }
-                digit_bases(total, before, tot_s, base_s);
-            }
-#pragma unroll
-            for (int rd = 0; rd < kSortMaxRounds; ++rd) {
-                if (rd < R) {
-                    const uint32_t e = first + rd * 32 + lane;
-                    if (e < k) {
-                        const uint32_t dd = ((kmax - skey[rd]) >> shift) & (kSortBins - 1);
-                        const uint32_t pos = base_s[dd] + counters[warp][dd] + (warp >= kWarps / 2 ? half_cnt[0][dd] : 0u) + srank[rd];
-                        if (last) {
-                            p.out_idx[pos] = sidx[rd];
-                            if (p.out_vals) p.out_vals[pos] = loss_of_key(skey[rd], losses, sidx[rd]);
-                        } else {
-                            cluster.map_shared_rank(pairs_out, pos >> tshift)[pos & tmask] = make_uint2(skey[rd], static_cast<uint32_t>(sidx[rd]));
-                        }
-                    }
-                }
-            }
-        }
-        if (!last) cluster.sync();  // after the last pass's exchange nobody touches another block's shared memory
     }
+    cluster.barrier_wait();  // no block exits while another may still read its shared memory
 }
 
 // Small pools: one CTA sorts all N composite keys (key, ~index), one per thread, with a
@@ -957,12 +1215,11 @@ cudaError_t launch_select(const SelectParams& p, int grid, cudaStream_t s) {
 
 // One cluster of `grid` blocks; it may be scheduled while the previous kernel of the stream drains (it waits for
 // that kernel's completion before its first global access).
-template <int CE, int CB>
-cudaLaunchConfig_t cluster_config(int grid, cudaStream_t s, cudaLaunchAttribute (&attr)[2]) {
+inline cudaLaunchConfig_t cluster_config(int grid, size_t smem, cudaStream_t s, cudaLaunchAttribute (&attr)[2]) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = ClusterLayout<CE, CB>::kSmemBytes;
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = static_cast<unsigned>(grid);
@@ -977,11 +1234,14 @@ cudaLaunchConfig_t cluster_config(int grid, cudaStream_t s, cudaLaunchAttribute 
 
 template <int CE, int CB>
 cudaError_t launch_cluster(const SelectParams& p, int grid, cudaStream_t s) {
-    cudaError_t e = allow_dynamic_smem(topk_cluster_kernel<CE, CB>, ClusterLayout<CE, CB>::kSmemBytes);
+    const bool sorted = p.order != LSGD_ORDER_INDEX_ASC;
+    auto kernel = sorted ? topk_cluster_sorted_kernel<CE, CB> : topk_cluster_kernel<CE, CB>;
+    const size_t smem = sorted ? SortedClusterLayout<CE, CB>::kSmemBytes : ClusterLayout<CE, CB>::kSmemBytes;
+    cudaError_t e = allow_dynamic_smem(kernel, smem);
     if (e != cudaSuccess) return e;
     cudaLaunchAttribute attr[2];
-    cudaLaunchConfig_t cfg = cluster_config<CE, CB>(grid, s, attr);
-    return cudaLaunchKernelEx(&cfg, topk_cluster_kernel<CE, CB>, p);
+    cudaLaunchConfig_t cfg = cluster_config(grid, smem, s, attr);
+    return cudaLaunchKernelEx(&cfg, kernel, p);
 }
 
 // Whether this device runs the 16-block cluster variant (clusters of more than 8 blocks are an opt-in, and the device
@@ -995,14 +1255,18 @@ bool wide_cluster_ok() {
     int& k = known[dev & 63];
     if (k == 0) {
         k = 2;
-        auto kernel = topk_cluster_kernel<4, 16>;
-        if (allow_dynamic_smem(kernel, ClusterLayout<4, 16>::kSmemBytes) == cudaSuccess &&
-            cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+        auto fits = [](auto kernel, size_t smem) {
+            if (allow_dynamic_smem(kernel, smem) != cudaSuccess ||
+                cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
+                return false;
             cudaLaunchAttribute attr[2];
-            cudaLaunchConfig_t cfg = cluster_config<4, 16>(16, nullptr, attr);
+            cudaLaunchConfig_t cfg = cluster_config(16, smem, nullptr, attr);
             int clusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg) == cudaSuccess && clusters >= 1) k = 1;
-        }
+            return cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg) == cudaSuccess && clusters >= 1;
+        };
+        if (fits(topk_cluster_kernel<4, 16>, ClusterLayout<4, 16>::kSmemBytes) &&
+            fits(topk_cluster_sorted_kernel<4, 16>, SortedClusterLayout<4, 16>::kSmemBytes))
+            k = 1;
         cudaGetLastError();  // a refusal above is an answer, not an error of the call being made
     }
     return k == 1;
