@@ -128,7 +128,7 @@ lsgd_status lsgd_score_losses(const void* logits, lsgd_dtype dtype, const int64_
     st = check_ws(ws, ws_bytes, score_workspace_bytes(N, T, C));
     if (st != LSGD_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(StatusBlock), s);
+    cudaError_t e = clear_device_words(ws, sizeof(StatusBlock), s);
     if (e != cudaSuccess) return LSGD_ERR_CUDA;
     return from_cuda(launch_score(logits, dtype, labels, N, T, C, ignore_index, losses, carve_score(ws, N, T, C),
                                   nullptr, s));

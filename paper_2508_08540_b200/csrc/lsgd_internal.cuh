@@ -93,11 +93,11 @@ int sm_count();  // multiprocessors of the current device (cached per device)
 // (programmatic dependent launch).  Such a kernel must call grid_dependency_wait() before it touches global
 // memory: that is where it waits for the previous kernel to have completed, with its writes visible.
 template <typename... KArgs, typename... Args>
-cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, cudaStream_t s, Args... args) {
+cudaError_t launch_dependent_smem(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t s, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
     cfg.blockDim = dim3(static_cast<unsigned>(block));
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -106,6 +106,15 @@ cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, cuda
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, cudaStream_t s, Args... args) {
+    return launch_dependent_smem(kernel, grid, block, 0, s, args...);
+}
+
+// Clears `bytes` (a multiple of 16, 16-byte aligned) of device memory with a kernel that lets the next kernel of the
+// stream start at once: a scorer launched with launch_dependent_smem reads its inputs while the head of the workspace
+// is still being cleared and waits (grid_dependency_wait) only before it first touches the status block or a histogram.
+cudaError_t clear_device_words(void* p, size_t bytes, cudaStream_t s);
 
 // ---------------------------------------------------------------------------
 // Device helpers

@@ -397,6 +397,7 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
 #pragma unroll
     for (int i = 0; i < kGroupStages - 1; ++i) issue(i);
     int64_t y = label_of(0);
+    grid_dependency_wait();  // the status block and the histogram are clear from here on (the first tiles are on their way)
     for (int64_t i = 0; i < my_tiles; ++i) {
         issue(i + kGroupStages - 1);
         const int64_t y_next = label_of(i + 1);
@@ -659,6 +660,7 @@ score_lane_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
         float loss = 0.f;
         if (cls == 2) {
             loss = __uint_as_float(0x7FC00000u);
+            grid_dependency_wait();  // the status block is clear from here on
             atomicAdd(&status->bad_labels, 1);
         } else if (cls == 0) {
             loss = loss_without_true_class(m, m * kLog2e, s, xy);
@@ -670,6 +672,7 @@ score_lane_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
     }
     cp_async_wait<0>();
     __syncthreads();
+    grid_dependency_wait();  // the workspace's histogram is clear from here on
     h.flush();
 }
 
@@ -952,9 +955,9 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
             }
             const int64_t want = ((rows + 31) / 32 + threads / 32 - 1) / (threads / 32);
             const int grid = static_cast<int>(std::min({want, static_cast<int64_t>(sms) * bps, max_ctas}));
-            kernel<<<grid, threads, smem, s>>>(logits, labels, rows, static_cast<int>(C), ignore_index, row_loss, status,
-                                               hist0, stage_bytes, head);
-            err = cudaGetLastError();
+            // may start while the head of the workspace is still being cleared (the kernel waits before it touches it)
+            err = launch_dependent_smem(kernel, grid, threads, smem, s, logits, labels, rows, static_cast<int>(C), ignore_index,
+                                        row_loss, status, hist0, stage_bytes, head);
         };
         if (C <= kTinyMaxC) {
             auto by_len = [&](auto cb_tag) {
@@ -1016,9 +1019,8 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
             }
             const int64_t tiles = (rows + tile_rows - 1) / tile_rows;
             const int grid = static_cast<int>(std::min({tiles, static_cast<int64_t>(sms) * bps, max_ctas}));
-            kernel<<<grid, kGroupThreads, smem, s>>>(logits, labels, rows, static_cast<int>(C), ignore_index, row_loss,
-                                                     status, hist0, stage_bytes);
-            err = cudaGetLastError();
+            err = launch_dependent_smem(kernel, grid, kGroupThreads, smem, s, logits, labels, rows, static_cast<int>(C), ignore_index,
+                                        row_loss, status, hist0, stage_bytes);
         };
         auto by_chunk = [&](auto lanes_tag, auto regs_tag) {
             constexpr int LN = decltype(lanes_tag)::value;

@@ -6,7 +6,8 @@
 // and the result is exact and bit-reproducible.
 //
 // One kernel does the whole selection, in phases separated by a barrier over all
-// its thread blocks:
+// its thread blocks.  Pools above 65,536 entries (topk_select_kernel, a cooperative
+// launch with one block per multiprocessor that exchanges through the workspace):
 //   1. radix select: three digit histograms (11 + 11 + 10 bits, most significant
 //      first; the first one may come ready-made from the scorer) find the key T of
 //      the k-th entry and r, the number of entries equal to T that still belong to
@@ -21,13 +22,15 @@
 //      if all selected keys are equal); stability turns the index-ascending input
 //      order into the required tie-break.  A pass is two phases: rank every tile
 //      by the digit (which gives the tile's digit counts), then scatter.
-// Pools of up to 65,536 entries run as ONE thread-block cluster that keeps all it
-// exchanges in distributed shared memory (topk_cluster_kernel: the barrier is the
-// cluster's hardware barrier); larger pools as a cooperative launch with one
-// block per multiprocessor that exchanges through the workspace (all blocks
-// resident by construction; the barrier is an arrival counter in the status
-// block, polled with a limit: if it ever ran out, the block would set the status
-// block's timeout word and return, and the other blocks would follow).
+//   All blocks are resident by construction; the barrier is an arrival counter in
+//   the status block, polled with a limit: if it ever ran out, the block would set
+//   the status block's timeout word and return, and the other blocks would follow.
+// Pools of up to 65,536 entries run as ONE thread-block cluster whose barrier is the
+// cluster's hardware barrier and which keeps its keys in registers and what blocks
+// exchange in distributed shared memory: topk_cluster_kernel (index-ascending
+// output: steps 1 to 3) and topk_cluster_sorted_kernel (loss-descending output:
+// two digits of step 1, then a sort of every key from the k-th key's bin upwards
+// with one barrier per pass; the first k sorted positions are the selection).
 // Pools of at most kSmallN entries are sorted whole by a single block instead.
 #include <cooperative_groups.h>
 
@@ -89,9 +92,21 @@ TopkWorkspace carve_topk(void* ws, int64_t N, int64_t k) {
     return w;
 }
 
-cudaError_t zero_topk_workspace(void* ws, int64_t k, cudaStream_t s) {
-    return cudaMemsetAsync(ws, 0, topk_zero_bytes(k), s);
+namespace {
+__global__ void clear_words_kernel(uint4* p, int n) {
+    grid_launch_dependents();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) p[i] = make_uint4(0u, 0u, 0u, 0u);
 }
+}  // namespace
+
+cudaError_t clear_device_words(void* p, size_t bytes, cudaStream_t s) {
+    const int n = static_cast<int>(bytes / 16);
+    clear_words_kernel<<<(n + 255) / 256, 256, 0, s>>>(static_cast<uint4*>(p), n);
+    return cudaGetLastError();
+}
+
+cudaError_t zero_topk_workspace(void* ws, int64_t k, cudaStream_t s) { return clear_device_words(ws, topk_zero_bytes(k), s); }
 
 namespace {
 

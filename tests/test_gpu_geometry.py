@@ -130,6 +130,48 @@ def test_selector_sort_pass_counts(L, oracle):
             np.testing.assert_array_equal(vals.cpu().numpy().view(np.uint32), want_vals.view(np.uint32))
 
 
+def test_selector_when_the_candidates_outnumber_the_selection(L, oracle):
+    """Loss-descending output of pools of up to 65,536 entries sorts every key that shares the k-th key's leading 22
+    bits or lies above them, and keeps the first k.  Pools where those candidates are far more than k, up to the
+    whole pool (every count then sits at the limit of the 16-bit halves the blocks exchange), in sorted and reversed
+    order (all candidates in the last or the first block), in the wide and the narrow cluster and without one."""
+    rng = np.random.default_rng(65)
+    N = 65_536
+    pools = {
+        "all equal": np.full(N, 1.75, np.float32),
+        "two values": np.where(rng.random(N) < 0.5, np.float32(2.0), np.float32(2.0000002)).astype(np.float32),
+        "37 values": rng.choice(rng.gamma(2.0, 1.0, 37).astype(np.float32), N),
+        "within 1024 keys": (np.float32(3.0).view(np.uint32) + rng.integers(0, 1024, N).astype(np.uint32)).view(np.float32),
+        "ascending": np.sort(rng.gamma(2.0, 1.0, N).astype(np.float32)),
+        "descending": np.sort(rng.gamma(2.0, 1.0, N).astype(np.float32))[::-1].copy(),
+    }
+    for name, h in pools.items():
+        v = torch.from_numpy(h).cuda()
+        for k in (1, 100, 16_384, 40_000, N):
+            want_idx, want_vals = oracle.topk(h, k, oracle.LOSS_DESC)
+            for kw in (dict(), dict(narrow_cluster=True), dict(no_cluster=True)):
+                with geometry(**kw):
+                    idx, vals = L.topk_select(v, k, L.ORDER_LOSS_DESC)
+                np.testing.assert_array_equal(idx.cpu().numpy(), want_idx, err_msg=f"{name} k={k} {kw}")
+                np.testing.assert_array_equal(vals.cpu().numpy().view(np.uint32), want_vals.view(np.uint32), err_msg=f"{name} k={k} {kw}")
+    # the same through the fused call (the scorer's histogram resolves the first digit): identical rows score identical bits
+    for N2, C in ((65_536, 10), (50_001, 7)):
+        row = rng.normal(0, 2, C).astype(np.float32)
+        x = np.tile(row, (N2, 1))
+        x[N2 // 3] += 1.0  # two rows that differ, so that the pool is not one value only
+        x[N2 - 5] -= 1.0
+        y = np.full((N2, 1), 3, np.int64)
+        d_x, d_y = torch.from_numpy(x).cuda().view(N2, 1, C), torch.from_numpy(y).cuda()
+        for k in (1, 3, 20_000, N2):
+            for kw in (dict(), dict(narrow_cluster=True)):
+                with geometry(**kw):
+                    losses, idx, vals = L.score_topk(d_x, d_y, k, L.ORDER_LOSS_DESC)
+                g = losses.cpu().numpy()
+                want_idx, want_vals = oracle.topk(g, k, oracle.LOSS_DESC)
+                np.testing.assert_array_equal(idx.cpu().numpy(), want_idx, err_msg=f"fused N={N2} k={k} {kw}")
+                np.testing.assert_array_equal(vals.cpu().numpy().view(np.uint32), want_vals.view(np.uint32))
+
+
 @pytest.mark.parametrize("N,T,C,dtype,k", [(20_000, 1, 100, "f32", 5_000), (300, 16, 5000, "bf16", 64), (70_000, 1, 10, "f32", 17_500)])
 def test_fused_call_is_the_same_in_every_geometry(L, oracle, N, T, C, dtype, k):
     x, y = pool(5, N, T, C, dtype, mask_p=0.1 if T > 1 else 0.0)
