@@ -223,6 +223,7 @@ __device__ void find_bin(const uint32_t* hist, int nbins, uint32_t& want, uint32
 
 // The same with two block barriers instead of five: every warp scans the warps' totals for itself.  `warp_tot` and
 // `result` must not be written again before another block barrier has been passed (none is taken at the end).
+// `result` holds three words; result[2] = the entries in the bin found.
 template <bool GLOBAL>
 __device__ __forceinline__ void find_bin_fast(const uint32_t* hist, int nbins, uint32_t& want, uint32_t& bin, uint32_t* warp_tot, uint32_t* result) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -251,6 +252,7 @@ __device__ __forceinline__ void find_bin_fast(const uint32_t* hist, int nbins, u
         const bool first = want <= before + c0;
         result[0] = first ? b0 : b0 - 1;
         result[1] = first ? want - before : want - before - c0;
+        result[2] = first ? c0 : c1;
     }
     __syncthreads();
     bin = result[0];
@@ -689,7 +691,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_cluster_kernel(const __grid_
     uint32_t* hist_s = reinterpret_cast<uint32_t*>(cl_smem);
     uint4* cta_cnt = reinterpret_cast<uint4*>(cl_smem + Lay::kHistBytes);
     __shared__ uint32_t warp_tot[kWarps + 1];
-    __shared__ uint32_t result[2];
+    __shared__ uint32_t result[3];
     __shared__ uint32_t red[2];
     cg::cluster_group cluster = cg::this_cluster();
     const int tid = threadIdx.x, lane = tid & 31;
@@ -774,7 +776,8 @@ __global__ void __launch_bounds__(kThreads, 1) topk_cluster_kernel(const __grid_
 
 // Loss-descending output.  The selection stops after two digits: every key that shares the 22 resolved bits with the
 // k-th key, or lies above them, is a candidate (k' >= k of them: k plus the few keys in the k-th key's bin of 1,024
-// consecutive keys).  The candidates are sorted whole, stably, by v = key - T (T = the lowest key of that bin) in
+// consecutive keys); after one digit already where that leaves at most 2 k candidates that fit the tiles k needs.
+// The candidates are sorted whole, stably, by v = key - T (T = the lowest key of that bin) in
 // descending 9-bit digits, least significant first; the first k positions of the result are the selection, ties
 // between equal keys in index order because the candidates start in index order.  No threshold has to be exact and
 // no tie has to be counted before the sort.
@@ -815,7 +818,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_cluster_sorted_kernel(const 
     uint32_t* flow = reinterpret_cast<uint32_t*>(cl_smem + Lay::kCountersBytes + Lay::kPairsBytes);  // [2][CB][kRowWords], two digits a word
     uint32_t* dig_hist = flow + kFlowWords;                                                          // [kDigits][kRowWords]
     __shared__ uint32_t warp_tot[kWarps + 1];
-    __shared__ uint32_t result[2];
+    __shared__ uint32_t result[3];
     __shared__ uint32_t vmax_s, vmax_all_s;
     __shared__ uint32_t warp_sum[kWarps];
     __shared__ uint32_t acc_s[2][kRowWords];  // sums of what is read from the other blocks, two digits a word: all of them; the blocks before this one
@@ -859,14 +862,23 @@ __global__ void __launch_bounds__(kThreads, 1) topk_cluster_sorted_kernel(const 
         key[i] = j < N ? loss_key(losses[j]) : 0u;
     }
 
-    // ---- 1. the two leading digits of the k-th key ----
+    // ---- 1. the leading digit of the k-th key, and the second one unless the first leaves few enough candidates ----
     uint32_t prefix = 0, want = p.k;
     if (p.hist0_ready) {
         uint32_t bin;
         find_bin_fast<true>(p.ws.hist, kSelBins, want, bin, warp_tot, result);
         prefix = bin << 21;
+    } else {
+        cluster_select_digits<CE>(cluster, key, 0, 0, hist_s, p.ws.hist, warp_tot, result, prefix, want);
     }
-    cluster_select_digits<CE>(cluster, key, p.hist0_ready ? 1 : 0, 1, hist_s, p.ws.hist, warp_tot, result, prefix, want);
+    {
+        // every key of the first digit's bin and above: if sorting them all needs no larger tiles than the selection
+        // itself and at most twice the entries, the second digit's exchange costs more than it saves
+        const uint32_t all = p.k - want + result[2];
+        uint32_t cap = nblocks * 1024u;
+        while (cap < p.k) cap <<= 1;
+        if (all > cap || all > 2 * p.k) cluster_select_digits<CE>(cluster, key, 1, 1, hist_s, p.ws.hist, warp_tot, result, prefix, want);
+    }
     const uint32_t T = prefix;  // candidates: key >= T (and a real key: padding is 0)
 
     // ---- 2. this block's digit histograms of v = key - T for all passes, its largest v, and each warp's

@@ -132,7 +132,7 @@ def test_selector_sort_pass_counts(L, oracle):
 
 def test_selector_when_the_candidates_outnumber_the_selection(L, oracle):
     """Loss-descending output of pools of up to 65,536 entries sorts every key that shares the k-th key's leading 22
-    bits or lies above them, and keeps the first k.  Pools where those candidates are far more than k, up to the
+    (or, where that leaves few enough, 11) bits or lies above them, and keeps the first k.  Pools where those candidates are far more than k, up to the
     whole pool (every count then sits at the limit of the 16-bit halves the blocks exchange), in sorted and reversed
     order (all candidates in the last or the first block), in the wide and the narrow cluster and without one."""
     rng = np.random.default_rng(65)
