@@ -493,8 +493,9 @@ def run_gpu(args, cfg):
 
 
 def launches_per_step(cfg) -> int:
-    """Kernels of liblsgd launched by one step (memsets excluded), from the launch logic of the library."""
-    n = 1 + (1 if cfg.T > 1 else 0)                # scorer (+ sequence mean)
+    """Kernels of liblsgd launched by one step, from the launch logic of the library."""
+    n = 1                                           # the kernel that clears the head of the workspace
+    n += 1 + (1 if cfg.T > 1 else 0)                # scorer (+ sequence mean)
     n += 1                                          # the selector is one kernel at every pool size
     n += 1                                          # aggregation
     return n

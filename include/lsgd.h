@@ -53,7 +53,7 @@ typedef enum lsgd_status {
     LSGD_ERR_UNSUPPORTED = 2, /* a dtype / order value the library does not know, N >= 2^31          */
     LSGD_ERR_ALIGNMENT = 3,   /* pointer not aligned to its element size, workspace not to 256 B      */
     LSGD_ERR_WORKSPACE = 4,   /* ws_bytes smaller than the matching *_workspace_bytes query           */
-    LSGD_ERR_CUDA = 5,        /* the CUDA runtime refused a launch or a memset                        */
+    LSGD_ERR_CUDA = 5,        /* the CUDA runtime refused a launch                                    */
     LSGD_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out (reported by lsgd_read_device_status)       */
 } lsgd_status;
 

@@ -11,7 +11,7 @@ namespace lsgd {
 
 // ---------------------------------------------------------------------------
 // Status block: the first 256 bytes of every scoring / selection workspace.
-// Zeroed (together with the selector's histograms) by one memset per call.
+// Zeroed (together with the selector's histograms) by one clearing kernel per call.
 // ---------------------------------------------------------------------------
 struct StatusBlock {
     int32_t bad_labels;      // tokens with a label outside [0, C) that is not ignore_index

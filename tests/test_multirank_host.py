@@ -50,9 +50,9 @@ def test_bench_accounting_helpers():
     b = bench.score_topk_bytes(cfg, labels)
     assert b == (cfg.N - 100) * (cfg.C * 4 + 4) + cfg.N * 8 + 4 * cfg.N + 8 * cfg.k
     assert bench.aggregate_bytes(cfg) == 4 * cfg.D * (cfg.P + 1)
-    assert bench.launches_per_step(wl.CONFIGS[4]) == 1 + 1 + 1 + 1
-    assert bench.launches_per_step(wl.CONFIGS[5]) == 1 + 1 + 1
-    assert bench.launches_per_step(wl.CONFIGS[1]) == 1 + 1 + 1
+    assert bench.launches_per_step(wl.CONFIGS[4]) == 1 + 1 + 1 + 1 + 1  # clear, scorer, sequence mean, selector, Eq. 3
+    assert bench.launches_per_step(wl.CONFIGS[5]) == 1 + 1 + 1 + 1
+    assert bench.launches_per_step(wl.CONFIGS[1]) == 1 + 1 + 1 + 1
 
 
 _RANK_STUB = """
