@@ -157,15 +157,15 @@ __device__ __forceinline__ bool grid_sync(StatusBlock* st, uint32_t& epoch, uint
         atomicAdd(&st->grid_arrivals, 1u);
         int ok = 1;
         uint32_t polls = 0;
+        // (the acquiring load orders this thread's later reads, the block barrier below those of the other threads)
         while (ld_acquire(&st->grid_arrivals) < target) {
             if (++polls > max_polls || ((polls & 63u) == 0 && *reinterpret_cast<volatile int32_t*>(&st->timeout) != 0)) {
                 ok = 0;
                 break;
             }
-            __nanosleep(32);
+            if (polls > 64u) __nanosleep(32);
         }
         if (!ok) atomicExch(&st->timeout, 1);
-        __threadfence();
         ok_s = ok;
     }
     __syncthreads();
@@ -200,32 +200,13 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* w
     return warp_tot[warp] + inc - v;
 }
 
-// Walks a finished histogram (global memory) from its highest bin down and finds the bin that holds the `want`-th
-// entry (1-based).  On return (all threads): bin, and `want` reduced by the entries in the bins above it.
-template <bool GLOBAL = true>
-__device__ void find_bin(const uint32_t* hist, int nbins, uint32_t& want, uint32_t& bin, uint32_t* warp_tot, uint32_t* result) {
-    // thread t owns bins nbins - 1 - 2 t and nbins - 2 - 2 t (or the single bin nbins - 1 - t), highest first
-    const bool two = nbins == 2 * kThreads;
-    const int b0 = two ? nbins - 1 - 2 * static_cast<int>(threadIdx.x) : nbins - 1 - static_cast<int>(threadIdx.x);
-    const uint32_t c0 = GLOBAL ? __ldcg(hist + b0) : hist[b0];
-    const uint32_t c1 = !two ? 0u : GLOBAL ? __ldcg(hist + b0 - 1) : hist[b0 - 1];
-    const uint32_t before = block_exclusive_scan(c0 + c1, warp_tot);
-    if (before < want && want <= before + c0 + c1) {
-        const bool first = want <= before + c0;
-        result[0] = first ? b0 : b0 - 1;
-        result[1] = first ? want - before : want - before - c0;
-    }
-    __syncthreads();
-    bin = result[0];
-    want = result[1];
-    __syncthreads();
-}
-
-// The same with two block barriers instead of five: every warp scans the warps' totals for itself.  `warp_tot` and
-// `result` must not be written again before another block barrier has been passed (none is taken at the end).
-// `result` holds three words; result[2] = the entries in the bin found.
+// Walks a finished histogram from its highest bin down and finds the bin that holds the `want`-th entry (1-based).
+// On return (all threads): bin, `want` reduced by the entries in the bins above it, and result[2] = the entries in
+// the bin found (`result` holds three words).  Two block barriers: every warp scans the warps' totals for itself.
+// `warp_tot` and `result` must not be written again before another block barrier has been passed (none is taken at
+// the end).
 template <bool GLOBAL>
-__device__ __forceinline__ void find_bin_fast(const uint32_t* hist, int nbins, uint32_t& want, uint32_t& bin, uint32_t* warp_tot, uint32_t* result) {
+__device__ __forceinline__ void find_bin(const uint32_t* hist, int nbins, uint32_t& want, uint32_t& bin, uint32_t* warp_tot, uint32_t* result) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool two = nbins == 2 * kThreads;
     const int b0 = two ? nbins - 1 - 2 * static_cast<int>(threadIdx.x) : nbins - 1 - static_cast<int>(threadIdx.x);
@@ -325,12 +306,13 @@ __device__ __forceinline__ uint32_t match_digit(uint32_t d, bool live) {
     return live ? peers : 0u;
 }
 
-// E: keys per thread of a selection tile (tiles of 1024 E entries; block b takes tiles b, b + gridDim.x, ...).
+// E: keys per thread of a selection tile (tiles of 1024 E entries, E = 4, 8, 12 or 16: the smallest that gives every
+// tile a block of its own; block b takes tiles b, b + gridDim.x, ...).
 template <int E>
 __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_constant__ SelectParams p) {
     extern __shared__ __align__(16) uint32_t dyn_smem[];  // selection: hist_s[kSelBins]; sort: counters[kWarps][kCounterPitch]
     __shared__ uint32_t warp_tot[kWarps + 1];
-    __shared__ uint32_t result[2];
+    __shared__ uint32_t result[3];
     __shared__ uint32_t red[3];
     __shared__ uint32_t part_tot[2][kSortBins], part_bef[2][kSortBins];
     __shared__ uint32_t base_s[kSortBins], tot_s[kSortBins], half_cnt[2][kSortBins];
@@ -364,7 +346,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
     uint32_t prefix = 0, want = p.k;
     if (p.hist0_ready) {
         uint32_t bin;
-        find_bin(p.ws.hist, kSelBins, want, bin, warp_tot, result);
+        find_bin<true>(p.ws.hist, kSelBins, want, bin, warp_tot, result);
         prefix = bin << 21;
     }
     for (int pass = p.hist0_ready ? 1 : 0; pass < kSelPasses; ++pass) {
@@ -388,7 +370,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
         }
         if (!grid_sync(status, epoch, p.barrier_parties, p.barrier_polls)) return;
         uint32_t bin;
-        find_bin(gh, pass == 2 ? 1024 : kSelBins, want, bin, warp_tot, result);
+        find_bin<true>(gh, pass == 2 ? 1024 : kSelBins, want, bin, warp_tot, result);
         prefix |= pass == 0 ? bin << 21 : pass == 1 ? bin << 10 : bin;
     }
     const uint32_t T = prefix, r = want;  // the k-th key, and how many entries equal to it are selected
@@ -624,8 +606,8 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
 // ---------------------------------------------------------------------------
 // Pools of up to 65,536 entries: ONE thread-block cluster, everything that blocks exchange kept in (distributed)
 // shared memory.  Block b owns a slice of 4,096 or 8,192 consecutive entries of the pool (in registers).  Digit
-// histograms of the selection are added into block 0's shared memory; block 0 resolves the digit and tells every
-// block.  The barrier is the cluster's hardware barrier.  Two kernels:
+// histograms of the selection are added up in the workspace (global atomics) and every block resolves the digit for
+// itself after one barrier.  The barrier is the cluster's hardware barrier.  Two kernels:
 //   topk_cluster_kernel         index-ascending output: exact threshold (three digits), per-block counts, ordered
 //                               compaction straight into the output;
 //   topk_cluster_sorted_kernel  loss-descending output: see there.
@@ -669,7 +651,7 @@ __device__ __forceinline__ void cluster_select_digits(cg::cluster_group& cluster
         }
         cluster.sync();  // every block's additions are in
         uint32_t bin;
-        find_bin_fast<true>(ghist + pass * kSelBins, pass == 2 ? 1024 : kSelBins, want, bin, warp_tot, result);
+        find_bin<true>(ghist + pass * kSelBins, pass == 2 ? 1024 : kSelBins, want, bin, warp_tot, result);
         prefix |= pass == 0 ? bin << 21 : pass == 1 ? bin << 10 : bin;
     }
 }
@@ -722,7 +704,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_cluster_kernel(const __grid_
     uint32_t prefix = 0, want = p.k;
     if (p.hist0_ready) {
         uint32_t bin;
-        find_bin_fast<true>(p.ws.hist, kSelBins, want, bin, warp_tot, result);
+        find_bin<true>(p.ws.hist, kSelBins, want, bin, warp_tot, result);
         prefix = bin << 21;
     }
     cluster_select_digits<kClE>(cluster, key, p.hist0_ready ? 1 : 0, kSelPasses - 1, hist_s, p.ws.hist, warp_tot, result, prefix, want);
@@ -866,7 +848,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_cluster_sorted_kernel(const 
     uint32_t prefix = 0, want = p.k;
     if (p.hist0_ready) {
         uint32_t bin;
-        find_bin_fast<true>(p.ws.hist, kSelBins, want, bin, warp_tot, result);
+        find_bin<true>(p.ws.hist, kSelBins, want, bin, warp_tot, result);
         prefix = bin << 21;
     } else {
         cluster_select_digits<CE>(cluster, key, 0, 0, hist_s, p.ws.hist, warp_tot, result, prefix, want);
@@ -1357,12 +1339,13 @@ cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order or
     p.sort_rounds = sort_rounds_for(k, std::min(resident, kSortDirectTiles));
     p.sort_tiles = static_cast<uint32_t>((k + 1024 * p.sort_rounds - 1) / (1024 * p.sort_rounds));
     auto tiles = [&](int e) { return (N + int64_t{kThreads} * e - 1) / (int64_t{kThreads} * e); };
-    const int e = tiles(4) <= resident ? 4 : tiles(8) <= resident ? 8 : 16;
+    const int e = tiles(4) <= resident ? 4 : tiles(8) <= resident ? 8 : tiles(12) <= resident ? 12 : 16;
     const int grid = static_cast<int>(std::min<int64_t>(resident, std::max<int64_t>(tiles(e), p.sort_tiles)));
     p.barrier_parties = static_cast<uint32_t>(grid) + (tg.phantom_block ? 1u : 0u);
     p.barrier_polls = tg.phantom_block ? 1u << 14 : kMaxPolls;
     if (e == 4) return launch_select<4>(p, grid, s);
     if (e == 8) return launch_select<8>(p, grid, s);
+    if (e == 12) return launch_select<12>(p, grid, s);
     return launch_select<16>(p, grid, s);
 }
 
