@@ -485,11 +485,79 @@ def run_gpu(args, cfg):
             "clocks": clocks.summary(),
             "input_generation_s": gen_s,
         }
+        if world == 1 and not args.no_other_configs and not (args.n_samples or args.d_params):
+            # the other four rounds, briefly, so that one run gives every configuration's figures from the same device
+            line["other_configs"] = {str(c): other_config_leg(wl.CONFIGS[c], dev, min(args.steps, 20), peak)
+                                     for c in sorted(wl.CONFIGS) if c != cfg.cfg_id}
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(cfg)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def other_config_leg(cfg, dev, steps: int, peak: float) -> dict:
+    """One of the other four rounds, timed briefly in the same process: the same two calls on that round's shapes,
+    inputs resident, L2 flushed before every step where the pool fits in it.  Mean and median over `steps` steps."""
+    import torch
+
+    from paper_2508_08540_b200 import lsgd
+
+    tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    d_logits = torch.empty((cfg.N, cfg.T, cfg.C), dtype=tdt, device=dev)
+    d_labels = torch.empty((cfg.N, cfg.T), dtype=torch.int64, device=dev)
+    es = d_logits.element_size()
+    slab = max(1, (1 << 28) // max(1, cfg.T * cfg.C * es))
+    unmasked = 0
+    for s0 in range(0, cfg.N, slab):
+        s1 = min(cfg.N, s0 + slab)
+        x, y = wl.pool_rows(cfg, s0, s1)
+        unmasked += int((y != wl.IGNORE_INDEX).sum())
+        hx = torch.from_numpy(x.view(np.int16)).view(torch.bfloat16) if cfg.dtype == "bf16" else torch.from_numpy(x)
+        d_logits[s0:s1].copy_(hx.reshape(s1 - s0, cfg.T, cfg.C))
+        d_labels[s0:s1].copy_(torch.from_numpy(y).reshape(s1 - s0, cfg.T))
+    d_reps = []
+    for i in range(cfg.P):
+        h = np.empty(cfg.D, dtype=np.float32)
+        wl.replica_slice(cfg, i, out=h)
+        d_reps.append(torch.from_numpy(h).to(dev))
+    weights = (lsgd.weights_from_steps(wl.step_counts(cfg).tolist()) if cfg.weight_mode == "steps"
+               else wl.weight_draws(cfg).tolist())
+    losses = torch.empty(cfg.N, dtype=torch.float32, device=dev)
+    idx = torch.empty(cfg.k, dtype=torch.int32, device=dev)
+    vals = torch.empty(cfg.k, dtype=torch.float32, device=dev)
+    out = torch.empty(cfg.D, dtype=torch.float32, device=dev)
+    ws = lsgd.workspace(lsgd.score_topk_workspace_bytes(cfg.N, cfg.T, cfg.C, cfg.k), dev)
+    flush = None if cfg.logit_bytes > (1 << 28) else torch.empty(1 << 28, dtype=torch.uint8, device=dev)
+    torch.cuda.synchronize()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    for i in range(3 + steps):
+        ev = evs[i - 3] if i >= 3 else None
+        if flush is not None:
+            flush.fill_(1)
+        if ev:
+            ev[0].record()
+        lsgd.score_topk(d_logits, d_labels, cfg.k, lsgd.ORDER_LOSS_DESC, losses=losses, out_idx=idx, out_vals=vals, ws=ws)
+        if ev:
+            ev[1].record()
+        lsgd.aggregate(d_reps, weights, out=out)
+        if ev:
+            ev[2].record()
+    torch.cuda.synchronize()
+    st = np.array([e[0].elapsed_time(e[1]) for e in evs])
+    ag = np.array([e[1].elapsed_time(e[2]) for e in evs])
+    st_bytes = unmasked * (cfg.C * es + 4) + cfg.N * cfg.T * 8 + 4 * cfg.N + 8 * cfg.k
+    ag_bytes = aggregate_bytes(cfg)
+    st_gbs = st_bytes / (st.mean() * 1e-3) / 1e9
+    ag_gbs = ag_bytes / (ag.mean() * 1e-3) / 1e9
+    return {"workload": workload_config(cfg)["workload"], "steps": steps, "l2": workload_config(cfg)["l2"],
+            "bad_labels": lsgd.read_device_status(ws),
+            "score_topk": {"samples_per_s": cfg.N / (st.mean() * 1e-3), "ms": float(st.mean()), "ms_median": float(np.median(st)),
+                           "gbs": st_gbs, "frac_of_measured_hbm": st_gbs / peak, "frac_of_nominal_8tbs": st_gbs / NOMINAL_HBM_GBS,
+                           "algorithmic_bytes": st_bytes},
+            "aggregation": {"ms": float(ag.mean()), "ms_median": float(np.median(ag)), "gbs": ag_gbs,
+                            "frac_of_measured_hbm": ag_gbs / peak, "frac_of_nominal_8tbs": ag_gbs / NOMINAL_HBM_GBS,
+                            "algorithmic_bytes": ag_bytes}}
 
 
 def launches_per_step(cfg) -> int:
@@ -600,6 +668,7 @@ def main():
     ap.add_argument("--sweep-scorer", action="store_true",
                     help="instead of the round: time lsgd_score_losses alone over a range of row lengths (1 GPU)")
     ap.add_argument("--sweep-filter", default="", help="with --sweep-scorer: only the row shape C:dtype[:rows]")
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the brief legs over the other four rounds")
     ap.add_argument("--no-round", action="store_true", help="skip the lsgd_aggregate_round legs (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--n-samples", type=int, default=0, help="profiling: shrink the pool to this many samples")
