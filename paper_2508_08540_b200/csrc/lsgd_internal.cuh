@@ -36,7 +36,7 @@ constexpr int kTile = 4096;               // smallest selection tile (the per-ti
 constexpr int kSmallN = 1024;             // pools up to this size are sorted by one CTA, one entry per thread
 constexpr int kSortBits = 9;              // digits of the stable LSD sort of the selected pairs
 constexpr int kSortBins = 1 << kSortBits;
-constexpr int kSortMaxRounds = 8;         // a sort tile holds 1024 R entries, R in {1, 2, 4, 8}
+constexpr int kSortMaxRounds = 8;         // a sort tile holds 1024 R entries, R from 1 to 8 (a power of two in the cluster kernels)
 constexpr int kSortDirectTiles = 256;     // the launcher grows R before it uses more sort tiles than this
 constexpr int kMaxClusterBlocks = 8;      // pools of up to 8 x 8,192 entries run as one cluster (of 16 x 4,096 where the device allows)
 

@@ -51,6 +51,13 @@ static int sort_rounds_for(int64_t k, int64_t max_tiles) {
         if ((k + 1024 * r - 1) / (1024 * r) <= max_tiles) return r;
     return kSortMaxRounds;
 }
+// The same for the cooperative kernel, whose tiles need not be a power of two: any R from 1 to 8 (k = 320,000 on 148
+// blocks: 105 tiles of 3,072 entries instead of 79 of 4,096).
+static int sort_rounds_any(int64_t k, int64_t max_tiles) {
+    for (int r = 1; r < kSortMaxRounds; ++r)
+        if ((k + 1024 * r - 1) / (1024 * r) <= max_tiles) return r;
+    return kSortMaxRounds;
+}
 // Upper bound of the number of sort tiles for any geometry the launcher may pick; grows with k, so that a
 // workspace sized for k also serves every smaller k.
 static size_t sort_tiles_bound(int64_t k) {
@@ -417,7 +424,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
     const uint32_t range = kmax - T;
     const int passes = p.order == LSGD_ORDER_INDEX_ASC ? 0 : (32 - __clz(range) + kSortBits - 1) / kSortBits;
     const bool direct = passes == 0;  // index order is the final order
-    const int tshift = 10 + (p.sort_rounds == 1 ? 0 : p.sort_rounds == 2 ? 1 : p.sort_rounds == 4 ? 2 : 3);
+    const uint32_t tile_entries = 1024u * static_cast<uint32_t>(p.sort_rounds);
     const uint32_t St = p.sort_tiles;
     for_each_tile([&](int64_t tile, const uint32_t (&key)[E]) {
         // entries above / equal to the threshold in the tiles before this one
@@ -496,7 +503,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
         // warps before w of the same half of the block, half_cnt[h][d] the count of half h.
         auto rank_tile = [&](uint32_t tile, bool publish) {
             for (int i = tid; i < kWarps * kCounterPitch; i += kThreads) dyn_smem[i] = 0;
-            const uint32_t first = (tile << tshift) + warp * (R * 32);
+            const uint32_t first = tile * tile_entries + warp * (R * 32);
 #pragma unroll
             for (int rd = 0; rd < kSortMaxRounds; ++rd) {  // all loads first: they are independent
                 const uint32_t e = first + rd * 32 + lane;
@@ -581,7 +588,7 @@ __global__ void __launch_bounds__(kThreads, 1) topk_select_kernel(const __grid_c
                 const bool mine = tid < kSortBins;
                 digit_bases(mine ? part_tot[0][tid] + part_tot[1][tid] : 0u, mine ? part_bef[0][tid] + part_bef[1][tid] : 0u, tot_s, base_s);
             }
-            const uint32_t first = (tile << tshift) + warp * (R * 32);
+            const uint32_t first = tile * tile_entries + warp * (R * 32);
 #pragma unroll
             for (int rd = 0; rd < kSortMaxRounds; ++rd) {
                 if (rd < R) {
@@ -1336,7 +1343,7 @@ cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order or
         if (ze != cudaSuccess) return ze;
     }
     const int resident = std::max(1, std::min(resident_blocks(), tg.max_ctas));
-    p.sort_rounds = sort_rounds_for(k, std::min(resident, kSortDirectTiles));
+    p.sort_rounds = sort_rounds_any(k, std::min(resident, kSortDirectTiles));
     p.sort_tiles = static_cast<uint32_t>((k + 1024 * p.sort_rounds - 1) / (1024 * p.sort_rounds));
     auto tiles = [&](int e) { return (N + int64_t{kThreads} * e - 1) / (int64_t{kThreads} * e); };
     const int e = tiles(4) <= resident ? 4 : tiles(8) <= resident ? 8 : tiles(12) <= resident ? 12 : 16;
