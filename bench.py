@@ -230,7 +230,7 @@ def job_throughput(world: int, units_per_rank: float, steps: int, ms: float) -> 
 # score_stream_rows_kernel or aggregate_vec4_kernel changes, until the counters have been taken again.
 NCU_TRAFFIC_BYTES = {
     ("score", 4): 7.27e9,      # 908.5 MB for 128 of 1,024 sequences
-    ("aggregate", 4): 4.77e9,  # 697.8 MB for 16,000,000 of 109,482,240 parameters
+    ("aggregate", 4): 4.77e9,  # 697.3 MB for 16,000,000 of 109,482,240 parameters
 }
 
 
