@@ -31,7 +31,9 @@
 // output: steps 1 to 3) and topk_cluster_sorted_kernel (loss-descending output:
 // two digits of step 1, then a sort of every key from the k-th key's bin upwards
 // with one barrier per pass; the first k sorted positions are the selection).
-// Pools of at most kSmallN entries are sorted whole by a single block instead.
+// Pools of at most kSmallN entries: loss-descending output by counting (small_rank_kernel: every entry counts the
+// entries that come before it, no sort); index-ascending output from a single block that sorts the pool whole to
+// find the k-th composite key (small_topk_kernel).
 #include <cooperative_groups.h>
 
 #include <algorithm>
@@ -1108,12 +1110,74 @@ __global__ void __launch_bounds__(kThreads, 1) topk_cluster_sorted_kernel(const 
     cluster.barrier_wait();  // no block exits while another may still read its shared memory
 }
 
-// Small pools: one CTA sorts all N composite keys (key, ~index), one per thread, with a
-// bitonic network; the first k are the selection in loss-descending order.
+// Small pools, loss-descending output: every entry finds its own position by counting, position = (entries with a
+// larger key) + (entries with the same key and a lower index), and writes itself there if that is below k.  No
+// sort and no exchange: each block keeps all N keys in shared memory (4 KB), a thread compares its key with four
+// others per shared-memory read (all lanes read the same address), and the few blocks run side by side on
+// different multiprocessors (N = 1,024: 8 blocks of 128 threads, about 2,300 instructions per thread, against 55
+// compare-exchange steps with 30 block barriers of the bitonic network below).
+constexpr int kRankThreads = 128;
+
+__global__ void __launch_bounds__(kRankThreads)
+small_rank_kernel(const float* __restrict__ losses, int n, int k, int32_t* __restrict__ out_idx,
+                  float* __restrict__ out_vals, StatusBlock* status) {
+    __shared__ __align__(16) uint32_t keys[kSmallN];
+    grid_dependency_wait();
+    if (status && blockIdx.x == 0 && threadIdx.x == 0) {  // a selection on its own: "nothing to report"
+        status->bad_labels = 0;
+        status->timeout = 0;
+    }
+    const int n4 = (n + 3) >> 2;
+#pragma unroll
+    for (int u = 0; u < kSmallN / kRankThreads; ++u) {  // (independent loads, all in flight at once)
+        const int j = u * kRankThreads + threadIdx.x;
+        if (j < 4 * n4) keys[j] = j < n ? loss_key(losses[j]) : 0u;  // key 0: below every loss
+    }
+    __syncthreads();
+    grid_launch_dependents();
+    const uint4* kv = reinterpret_cast<const uint4*>(keys);
+    for (int i = blockIdx.x * kRankThreads + threadIdx.x; i < n; i += gridDim.x * kRankThreads) {
+        const uint32_t me = keys[i];
+        const int ci = i >> 2;
+        uint32_t r0 = 0, r1 = 0, r2 = 0, r3 = 0;
+#pragma unroll 8
+        for (int c = 0; c < ci; ++c) {  // lower indices: equal keys come first
+            const uint4 q = kv[c];
+            r0 += q.x >= me;
+            r1 += q.y >= me;
+            r2 += q.z >= me;
+            r3 += q.w >= me;
+        }
+        {
+            const uint4 q = kv[ci];
+            const int e = i & 3;
+            r0 += e > 0 ? q.x >= me : false;
+            r1 += e > 1 ? q.y >= me : (e < 1 && q.y > me);
+            r2 += e > 2 ? q.z >= me : (e < 2 && q.z > me);
+            r3 += e < 3 && q.w > me;
+        }
+#pragma unroll 8
+        for (int c = ci + 1; c < n4; ++c) {  // higher indices: only larger keys come first
+            const uint4 q = kv[c];
+            r0 += q.x > me;
+            r1 += q.y > me;
+            r2 += q.z > me;
+            r3 += q.w > me;
+        }
+        const uint32_t pos = (r0 + r1) + (r2 + r3);
+        if (pos < static_cast<uint32_t>(k)) {
+            out_idx[pos] = i;
+            if (out_vals) out_vals[pos] = losses[i];
+        }
+    }
+}
+
+// Small pools, index-ascending output: one CTA sorts all N composite keys (key, ~index), one per thread, with a
+// bitonic network; the k-th of them is the cut, and the entries at or above it are written in index order.
 constexpr int kSmallThreads = 1024;
 
 __global__ void __launch_bounds__(kSmallThreads)
-small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int32_t* __restrict__ out_idx,
+small_topk_kernel(const float* __restrict__ losses, int n, int k, int32_t* __restrict__ out_idx,
                   float* __restrict__ out_vals, StatusBlock* status) {
     __shared__ unsigned long long ck[kSmallN];
     __shared__ uint32_t warp_tot[kSmallThreads / 32];
@@ -1156,15 +1220,7 @@ small_topk_kernel(const float* __restrict__ losses, int n, int k, int order, int
         __syncthreads();
     }
     grid_launch_dependents();
-    if (order == LSGD_ORDER_LOSS_DESC) {
-        for (int j = threadIdx.x; j < k; j += kSmallThreads) {
-            const int32_t i = static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(ck[j]));
-            out_idx[j] = i;
-            if (out_vals) out_vals[j] = losses[i];
-        }
-        return;
-    }
-    // index-ascending: an entry is selected iff its composite key is >= the k-th largest
+    // an entry is selected iff its composite key is >= the k-th largest
     const unsigned long long cut = ck[k - 1];
     const int j = threadIdx.x;  // one index per thread
     const bool sel = j < n && ((static_cast<unsigned long long>(loss_key(losses[j])) << 32) | (0xFFFFFFFFu - static_cast<uint32_t>(j))) >= cut;
@@ -1309,9 +1365,15 @@ int resident_blocks() {
 
 cudaError_t launch_topk(const float* losses, int64_t N, int64_t k, lsgd_order order, int32_t* out_idx,
                         float* out_vals, const TopkWorkspace& ws, bool hist0_ready, bool standalone, cudaStream_t s) {
-    if (N <= kSmallN)
+    if (N <= kSmallN) {
+        if (order == LSGD_ORDER_LOSS_DESC) {
+            const int grid = static_cast<int>(std::min<int64_t>((N + kRankThreads - 1) / kRankThreads, test_geometry().max_ctas));
+            return launch_dependent(small_rank_kernel, grid, kRankThreads, s, losses, static_cast<int>(N), static_cast<int>(k),
+                                    out_idx, out_vals, standalone ? ws.status : nullptr);
+        }
         return launch_dependent(small_topk_kernel, 1, kSmallThreads, s, losses, static_cast<int>(N), static_cast<int>(k),
-                                static_cast<int>(order), out_idx, out_vals, standalone ? ws.status : nullptr);
+                                out_idx, out_vals, standalone ? ws.status : nullptr);
+    }
     SelectParams p;
     p.losses = losses;
     p.N = N;
