@@ -623,7 +623,8 @@ def run_scorer_sweep(args):
         nbytes = rows * (C * x.element_size() + 12)
         out.append({"rows": rows, "C": C, "dtype": dt, "true_class_bump": bump, "row_bytes": C * x.element_size(), "ms": ms,
                     "gbs": nbytes / ms / 1e6, "frac_of_measured_hbm": nbytes / ms / 1e6 / peak})
-        del x, y, losses
+        del x, y, losses, ws
+        torch.cuda.empty_cache()  # every shape starts from freshly mapped memory
     print(json.dumps({"metric": "scorer GB/s by row shape", "unit": "GB/s", "peak": peak, "peak_source": peak_src,
                       "steps": args.steps, "data": "synthetic", "shapes": out}), flush=True)
 
