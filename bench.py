@@ -550,8 +550,11 @@ def other_config_leg(cfg, dev, steps: int, peak: float) -> dict:
     ag_bytes = aggregate_bytes(cfg)
     st_gbs = st_bytes / (st.mean() * 1e-3) / 1e9
     ag_gbs = ag_bytes / (ag.mean() * 1e-3) / 1e9
+    bad = lsgd.read_device_status(ws)
+    del d_logits, d_labels, d_reps, losses, idx, vals, out, ws, flush
+    torch.cuda.empty_cache()  # the next round's buffers are mapped afresh, not carved out of this round's
     return {"workload": workload_config(cfg)["workload"], "steps": steps, "l2": workload_config(cfg)["l2"],
-            "bad_labels": lsgd.read_device_status(ws),
+            "bad_labels": bad,
             "score_topk": {"samples_per_s": cfg.N / (st.mean() * 1e-3), "ms": float(st.mean()), "ms_median": float(np.median(st)),
                            "gbs": st_gbs, "frac_of_measured_hbm": st_gbs / peak, "frac_of_nominal_8tbs": st_gbs / NOMINAL_HBM_GBS,
                            "algorithmic_bytes": st_bytes},

@@ -604,7 +604,9 @@ score_lane_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict__
     // instruction stream is the limit (same run, of the copy rate: bf16 rows of 400 bytes 0.79 -> 0.87, of 100 bytes
     // 0.73 -> 0.77; fp32 rows of 40 bytes 0.80 -> 0.82, of 408 bytes 0.97 -> 1.05) and costs where memory is (fp32
     // rows of 400 bytes, whole chunks: 1.04 -> 0.97), so whole-chunk fp32 rows keep the 16-byte copies.
-    const bool flat = !PADDED ? true : (ES == 2 && CMAX == 0 ? (rc & 1) != 0 : false);  // (a constant in all but one case)
+    // (fp32 rows read element by element lost too: C = 101 0.86 -> 0.78.)
+    const bool flat = !PADDED ? !(ES == 4 && CMAX == 0 && CB == 4)
+                              : (ES == 2 && CMAX == 0 ? (rc & 1) != 0 : false);  // (a constant in all but one case)
     uint64_t* bars = reinterpret_cast<uint64_t*>(lane_smem + (hist0 ? kSelBins * sizeof(uint32_t) : 0) +
                                                  static_cast<size_t>(kWarpsPerCta) * STAGES * stage_bytes) + warp * STAGES;
     const int64_t blocks = (rows + 31) >> 5;
@@ -1128,14 +1130,14 @@ cudaError_t launch_rows(const T* logits, const int64_t* labels, int64_t rows, in
                 if constexpr (sizeof(T) == 2) go(score_group_rows_kernel<T, LN, 4, RG>, LN);  // (4-byte chunks of fp32 are single elements)
             } else go(score_group_rows_kernel<T, LN, 0, false>, LN);
         };
-        // rows per tile (128 / L) times bytes per row: at most 32 KB per stage (32 x 800, 16 x 2048, 8 x 2048), plus padding.
+        // rows per tile (128 / L) times bytes per row: at most 34 KB per stage (32 x 1024 at the padded pitch, 16 x 2048, 8 x 2048).
         // As few lanes per row as the row length allows: the per-row work is shared by the 32 / L rows of a warp.
         // Measured in one run, fraction of the copy rate: 600 and 800 bytes, 4 lanes 0.74-0.98 against 0.61-0.96 with
         // 8; 1000 bytes, 8 lanes (share in registers) 0.74 against 0.64 with 4 and 0.67 with 8 looping; 1280-1600
         // bytes, 8 lanes looping 0.86-1.02 against 0.71-0.97 with 16; 2000 bytes, fp32 1.00 with 8 lanes looping against
         // 0.94 with 16, bf16 (twice the elements per byte) 0.71 against 0.79.
         const bool vec = cb >= 8 || (cb == 4 && sizeof(T) == 2);
-        if (row_bytes <= 800) by_chunk(std::integral_constant<int, 4>{}, std::false_type{});
+        if (row_bytes <= (sizeof(T) == 4 ? 1024 : 800)) by_chunk(std::integral_constant<int, 4>{}, std::false_type{});  // (fp32 1,024 bytes: 1.01 with 4 lanes, 0.97 with 8; bf16 0.79 against 0.86)
         else if (row_bytes <= 1024) by_chunk(std::integral_constant<int, 8>{}, std::true_type{});
         else if (row_bytes <= (sizeof(T) == 4 ? 2048 : 1792) && vec) by_chunk(std::integral_constant<int, 8>{}, std::false_type{});
         else by_chunk(std::integral_constant<int, 16>{}, std::true_type{});
