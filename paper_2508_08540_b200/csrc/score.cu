@@ -445,19 +445,21 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
             if (mbar_try_wait(bar, parity)) return true;
         return false;
     };
-    auto label_of = [&](int64_t i) -> int64_t {
-        if (i >= my_tiles) return ignore_index;
-        const int64_t row = (blockIdx.x + i * gridDim.x) * R + g;
+    auto label_at = [&](int64_t row) -> int64_t {  // (a tile past this CTA's last one starts past the pool's end)
         return row < rows ? labels[row] : ignore_index;
     };
 
 #pragma unroll
     for (int i = 0; i < kGroupStages - 1; ++i) issue(i);
-    int64_t y = label_of(0);
+    int64_t y = label_at(static_cast<int64_t>(blockIdx.x) * R + g);
+    // every tile starts at the same offset from a 16-byte boundary (a tile's rows are a multiple of 16 bytes)
+    const int head = static_cast<int>(reinterpret_cast<uintptr_t>(logits) & 15);
+    const int64_t row_step = static_cast<int64_t>(gridDim.x) * R;
+    int64_t row_use = static_cast<int64_t>(blockIdx.x) * R;
     grid_dependency_wait();  // the status block and the histogram are clear from here on (the first tiles are on their way)
     for (int64_t i = 0; i < my_tiles; ++i) {
         issue(i + kGroupStages - 1);
-        const int64_t y_next = label_of(i + 1);
+        const int64_t y_next = label_at(row_use + row_step + g);
         if constexpr (PADDED) {
             cp_async_wait<kGroupStages - 1>();
             __syncthreads();  // everybody's copies of tile i have landed
@@ -467,9 +469,9 @@ score_group_rows_kernel(const T* __restrict__ logits, const int64_t* __restrict_
             if (i + 1 < my_tiles) landed(i + 1);
             break;
         }
-        const int64_t row0 = (blockIdx.x + i * gridDim.x) * R;
+        const int64_t row0 = row_use;  // (blockIdx.x + i gridDim.x) R, kept as a running sum
+        row_use += row_step;
         const bool mine = row0 + g < rows;
-        const int head = static_cast<int>((reinterpret_cast<uintptr_t>(logits) + row0 * row_bytes) & 15);
         unsigned char* buf = stages + (i % kGroupStages) * stage_bytes;
         const int cls = mine ? label_class(y, C, ignore_index) : 1;
         T* x = reinterpret_cast<T*>(buf + head + g * pitch_bytes);
