@@ -461,7 +461,7 @@ def run_gpu(args, cfg):
                             "algorithmic_bytes": ag_bytes},
             "warm": warm,
             "round_samples_per_s": world * cfg.N * args.steps / (total_ms * 1e-3),
-            "roofline": {"bound": "hbm", "kernel": "lsgd_score_topk (scorer kernel + memset, sequence mean, selector)",
+            "roofline": {"bound": "hbm", "kernel": "lsgd_score_topk (clearing kernel, scorer kernel, sequence mean, selector)",
                          "achieved": st_gbs, "peak": peak, "unit": "GB/s", "frac": st_gbs / peak,
                          "traffic": NCU_TRAFFIC_BYTES.get(("score", cfg.cfg_id)) if not (args.n_samples or args.d_params) else None,
                          "peak_source": peak_src},
