@@ -64,7 +64,7 @@ def aggregate_bytes(cfg) -> int:
 # clocks (read-only NVML sampling while the timed region runs)
 # --------------------------------------------------------------------------- #
 class ClockSampler:
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.003):
         self.samples, self.reasons, self.sm_max = [], set(), None
         self._stop = threading.Event()
         self._t = None
